@@ -1,0 +1,172 @@
+/*
+ * bls.h - C ABI of the B200 bounded-lag-synchronous (BLS) embedding lookup.
+ *
+ * One GPU emulates P logical ranks.  Every rank owns a partition of T embedding
+ * tables (all resident in device memory) and a row block of b = B/P samples of
+ * the batch.  One iteration of the path is
+ *   (1) route   every rank sorts the row IDs it needs by owner rank: alltoallv
+ *               send counts / displacements and a stably packed send buffer;
+ *   (2) lookup  every owner gathers the requested rows and sum-pools them per
+ *               bag with fp32 accumulation;
+ *   (3) return  the pooled vectors are written straight into the requester's
+ *               output layout out[src][s][t][:];
+ * and iterations are kept in a ring of k_max+1 slots driven by per-rank
+ * progress counters in device memory, so that ranks may be up to k iterations
+ * apart.
+ *
+ * Conventions
+ *   - All `const void*`/`int32_t*` data arguments are DEVICE pointers unless the
+ *     argument is documented as "host".  The library allocates no device
+ *     memory: the caller provides one workspace (bls_plan_bytes) and keeps
+ *     tables, workspace and per-iteration inputs alive as documented.
+ *   - All work is enqueued on the CUDA stream given to bls_plan; calls return
+ *     without synchronising unless stated.
+ *   - Bags are ordered (src, t, s): flat bag index g = (src*T + t)*b + s.
+ *     `offsets` is int32 [P*T*b + 1], exclusive prefix of bag lengths starting
+ *     at 0; `ids` is int32 [offsets[last]], row numbers into table t.
+ *   - Errors are return codes.  Conditions detected on the device (bad ID,
+ *     capacity exceeded, bounded wait expired) are latched in a device status
+ *     word and reported by bls_status(); the device never traps.
+ */
+#ifndef BLS_H
+#define BLS_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct bls_plan bls_plan_t;          /* opaque, host memory */
+
+typedef enum {
+    BLS_OK = 0,
+    BLS_EINVAL = 1,     /* bad argument / malformed offsets */
+    BLS_ENOSPC = 2,     /* workspace or per-rank ID capacity too small */
+    BLS_ECUDA = 3,      /* a CUDA runtime call failed */
+    BLS_ERANGE = 4,     /* an ID outside [0, rows) was seen (it was replaced by row 0) */
+    BLS_ETIMEOUT = 5,   /* a bounded device-side wait gave up */
+    BLS_ESTATE = 6      /* call order violated, k > k_max, or k changed mid-flight */
+} bls_status_t;
+
+typedef enum { BLS_F32 = 0, BLS_BF16 = 1, BLS_F16 = 2 } bls_dtype_t;
+
+/* Table placement ("a given partitioning strategy", Section I):
+ *   TABLE_RR   owner(t, id) = t mod P, owner-local row = id
+ *   ROW_BLOCK  owner(t, id) = id / ceil(rows_t / P), owner-local row = id - owner*ceil(rows_t/P) */
+typedef enum { BLS_PART_TABLE_RR = 0, BLS_PART_ROW_BLOCK = 1 } bls_part_t;
+
+/* One embedding table: row-major [rows][dim] of `dtype`, device memory, base
+ * 16-byte aligned, dim*sizeof(dtype) one of 16,32,64,128,256,512 bytes.  All
+ * tables of a plan share dim and dtype.  Borrowed for the plan's lifetime. */
+typedef struct {
+    const void *weight;
+    int64_t rows;
+    int32_t dim;
+    int32_t dtype;               /* bls_dtype_t */
+} bls_table_t;
+
+/* Device pointers to the routing artefacts and output of one iteration's slot
+ * (for parity checks and for consumers of the output).
+ *   sendcounts/sdispls  [P][P] indexed [src][dst]   (alltoallv arguments of the request leg)
+ *   recvcounts/rdispls  [P][P] indexed [dst][src]   (valid once the iteration has been looked up)
+ *   sendbuf             rank src's packed send buffer starts at sendbuf + src*sendbuf_stride;
+ *                       owner-local rows, sorted by dst, ties in original order
+ *   sub_start           rank src's array starts at sub_start + src*sub_stride and has
+ *                       subbags_per_rank + 1 entries: start position (in src's send buffer) of
+ *                       each sub-bag, ordered (dst, table, sample); consecutive differences are the
+ *                       sub-bag lengths the owner uses to rebuild bag boundaries
+ *   out                 fp32 [P][b][T][dim], the requester layout */
+typedef struct {
+    const int32_t *sendcounts, *sdispls, *recvcounts, *rdispls;
+    const int32_t *sendbuf;
+    int64_t sendbuf_stride;
+    const int32_t *sub_start;
+    int64_t sub_stride;
+    int64_t subbags_per_rank;
+    const float *out;
+} bls_route_view_t;
+
+/* ---- plan (Section III-B "Initialisation": buffers are created and registered
+ * once and then reused circularly; the bound is passed at initialisation) ---- */
+
+/* Workspace size in bytes for the given shape.  host call, no GPU work.
+ * max_ids_per_rank: capacity of one rank's send buffer (IDs per rank per iteration). */
+bls_status_t bls_plan_bytes(const bls_table_t *tables /*host*/, int T, int part, int P,
+                            int local_batch, int k_max, int64_t max_ids_per_rank, size_t *bytes /*host*/);
+
+/* Build a plan inside `workspace` (device, 256-byte aligned, `bytes` long, borrowed
+ * until bls_destroy).  Enqueues the initialisation of counters and descriptors on
+ * `cuda_stream` (a cudaStream_t; NULL = default stream).  P <= 32, k_max <= 15. */
+bls_status_t bls_plan(const bls_table_t *tables /*host*/, int T, int part, int P, int local_batch,
+                      int k_max, int64_t max_ids_per_rank, void *workspace, size_t bytes,
+                      void *cuda_stream, bls_plan_t **plan /*host out*/);
+
+void bls_destroy(bls_plan_t *plan);          /* frees host memory only; does not synchronise */
+
+/* ---- the synchronous decomposition (bound 0 == plain alltoallv, Section III-D) ----
+ * bls_route:  step (1) for every rank for iteration `iter` (must be the next
+ *             unissued iteration, with nothing outstanding).  ids/offsets are
+ *             borrowed until the call's work has run.
+ * bls_lookup: steps (2)+(3) for that iteration; afterwards bls_view(iter).out
+ *             holds the result until the next iteration is issued. */
+bls_status_t bls_route(bls_plan_t *plan, int64_t iter, const int32_t *ids, const int32_t *offsets,
+                       int64_t n_ids);
+bls_status_t bls_lookup(bls_plan_t *plan, int64_t iter);
+
+/* ---- the BLS loop (Section IV, Listing 2) ----
+ * bls_step: issue the next iteration t with bound k (0 <= k <= k_max, the same k
+ *           until everything outstanding has been drained).  Ranks that are not
+ *           held back by an injected stall route, serve and complete whatever
+ *           the counters allow; the call makes sure iteration t-k is complete on
+ *           every rank (the oldest request is waited for once more than k are
+ *           outstanding) and hands it back: *out = its fp32 [P][b][T][dim] block
+ *           inside the ring, *out_iter = t-k; or *out = NULL, *out_iter = -1
+ *           while t < k.  `*out` stays valid until the next bls_step/bls_drain
+ *           call on the stream.  ids/offsets of iteration t are borrowed until
+ *           k further steps (or the drain) have run.
+ * bls_drain: Listing 2's final loop, one outstanding iteration per call, oldest
+ *           first; *out = NULL once nothing is outstanding. */
+bls_status_t bls_step(bls_plan_t *plan, int k, const int32_t *ids, const int32_t *offsets,
+                      int64_t n_ids, const float **out /*host out*/, int64_t *out_iter /*host out*/);
+bls_status_t bls_drain(bls_plan_t *plan, const float **out /*host out*/, int64_t *out_iter /*host out*/);
+
+/* The same two calls with HOST input and output buffers: ids/offsets are copied
+ * to a staging area of the ring (pinned memory recommended), and the iteration
+ * handed back, if any, is copied to host_out (fp32 [P][b][T][dim]; may be NULL to
+ * skip the copy).  Copies are asynchronous on the plan's stream. */
+bls_status_t bls_step_host(bls_plan_t *plan, int k, const int32_t *ids /*host*/,
+                           const int32_t *offsets /*host*/, int64_t n_ids,
+                           float *host_out /*host*/, int64_t *out_iter /*host out*/);
+bls_status_t bls_drain_host(bls_plan_t *plan, float *host_out /*host*/, int64_t *out_iter /*host out*/);
+
+/* ---- inspection ---- */
+/* Device pointers of the slot that holds iteration `iter` (must still be in the ring). */
+bls_status_t bls_view(bls_plan_t *plan, int64_t iter, bls_route_view_t *view /*host out*/);
+/* Synchronises the stream; copies the P per-rank counters to host arrays (may be NULL). */
+bls_status_t bls_counters(bls_plan_t *plan, int64_t *posted, int64_t *served, int64_t *done);
+/* Synchronises the stream and returns the first latched device condition (BLS_OK if none);
+ * *max_lag (may be NULL) receives the largest distance ever seen between the newest
+ * posted iteration and the oldest incomplete one. */
+bls_status_t bls_status(bls_plan_t *plan, int64_t *max_lag /*host out*/);
+/* Injected delay of rank `rank` before each of its iterations (Section V-E,
+ * setting 2: a delay models a slowdown of any nature), in nanoseconds. */
+bls_status_t bls_set_stall(bls_plan_t *plan, int rank, int64_t ns);
+/* Upper limit of any single device-side wait (default 2 s). */
+bls_status_t bls_set_wait_limit(bls_plan_t *plan, int64_t ns);
+
+const char *bls_strerror(int status);
+
+/* ---- input generation helper (not part of the method) ----
+ * Fill rows [0, rows) of table `t` with the counter-hash values used by the
+ * synthetic workloads: SplitMix64 output number (t<<48 | row<<16 | c) + 1 for
+ * `seed`, four 16-bit fields summed, minus 131070, times 1/sqrt((65536^2-1)/3)
+ * in fp32, rounded to nearest even into `dtype`. */
+bls_status_t bls_fill_hash_table(void *weight, int64_t rows, int32_t dim, int32_t dtype,
+                                 uint64_t seed, int32_t t, void *cuda_stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* BLS_H */

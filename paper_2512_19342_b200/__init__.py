@@ -1,0 +1,9 @@
+"""B200-native bounded-lag-synchronous (BLS) embedding lookup.
+
+The product is the CUDA library ``libbls.so`` (sources under ``csrc/``, C ABI in
+``include/bls.h``); this package is its thin Python binding.
+"""
+from .binding import (BLS_OK, BLS_EINVAL, BLS_ENOSPC, BLS_ECUDA, BLS_ERANGE, BLS_ETIMEOUT, BLS_ESTATE,  # noqa: F401
+                      BlsError, Plan, bls_plan_bytes, bls_plan, bls_route, bls_lookup, bls_step,
+                      bls_drain, bls_step_host, bls_drain_host, bls_view, bls_counters, bls_status,
+                      bls_set_stall, bls_set_wait_limit, bls_fill_hash_table, lib, EXPORTS)

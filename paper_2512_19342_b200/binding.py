@@ -1,0 +1,214 @@
+"""Thin ctypes binding of ``libbls.so``: argument marshalling only.
+
+Every step of the path runs inside the CUDA library; torch is used here for
+device memory (workspace, tables, inputs) and for the current stream.  There is
+no CPU fallback: if the shared library is missing the first call raises.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import List, Optional, Sequence, Tuple
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libbls.so")
+
+BLS_OK, BLS_EINVAL, BLS_ENOSPC, BLS_ECUDA, BLS_ERANGE, BLS_ETIMEOUT, BLS_ESTATE = range(7)
+BLS_F32, BLS_BF16, BLS_F16 = 0, 1, 2
+BLS_PART_TABLE_RR, BLS_PART_ROW_BLOCK = 0, 1
+PART = {"table_rr": BLS_PART_TABLE_RR, "row_block": BLS_PART_ROW_BLOCK}
+_DTYPE = {torch.float32: BLS_F32, torch.bfloat16: BLS_BF16, torch.float16: BLS_F16}
+
+EXPORTS = ["bls_plan_bytes", "bls_plan", "bls_destroy", "bls_route", "bls_lookup", "bls_step",
+           "bls_drain", "bls_step_host", "bls_drain_host", "bls_view", "bls_counters", "bls_status",
+           "bls_set_stall", "bls_set_wait_limit", "bls_strerror", "bls_fill_hash_table"]
+
+
+class BlsError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        self.code = code
+        super().__init__(f"{where}: {lib().bls_strerror(code).decode()} (status {code})")
+
+
+class _Table(C.Structure):
+    _fields_ = [("weight", C.c_void_p), ("rows", C.c_int64), ("dim", C.c_int32), ("dtype", C.c_int32)]
+
+
+class _View(C.Structure):
+    _fields_ = [("sendcounts", C.c_void_p), ("sdispls", C.c_void_p), ("recvcounts", C.c_void_p),
+                ("rdispls", C.c_void_p), ("sendbuf", C.c_void_p), ("sendbuf_stride", C.c_int64),
+                ("sub_start", C.c_void_p), ("sub_stride", C.c_int64), ("subbags_per_rank", C.c_int64),
+                ("out", C.c_void_p)]
+
+
+_lib = None
+
+
+def lib():
+    """Load the CUDA library; fails loudly when it has not been built."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(f"{LIB_PATH} is missing: build it with `python -m paper_2512_19342_b200.build` "
+                               "(there is no CPU fallback)")
+        _lib = C.CDLL(LIB_PATH)
+        _lib.bls_strerror.restype = C.c_char_p
+        _lib.bls_strerror.argtypes = [C.c_int]
+    return _lib
+
+
+def _check(code: int, where: str):
+    if code != BLS_OK:
+        raise BlsError(code, where)
+
+
+def _stream_ptr(stream: Optional[torch.cuda.Stream]) -> C.c_void_p:
+    s = stream if stream is not None else torch.cuda.current_stream()
+    return C.c_void_p(s.cuda_stream)
+
+
+def _table_array(tables: Sequence[torch.Tensor]):
+    arr = (_Table * len(tables))()
+    for i, w in enumerate(tables):
+        if w.dim() != 2 or not w.is_contiguous():
+            raise ValueError("tables must be contiguous 2-D tensors")
+        arr[i] = _Table(w.data_ptr(), w.shape[0], w.shape[1], _DTYPE[w.dtype])
+    return arr
+
+
+class Plan:
+    """Handle of a plan plus the tensors it borrows (kept alive here)."""
+
+    def __init__(self, handle, tables, workspace, P, T, b, D, k_max, part, stream):
+        self.handle, self.tables, self.workspace = handle, list(tables), workspace
+        self.P, self.T, self.b, self.D, self.k_max, self.part = P, T, b, D, k_max, part
+        self.stream = stream
+        self._borrowed: List[Tuple[torch.Tensor, torch.Tensor]] = []
+
+    def _keep(self, ids, offsets):
+        self._borrowed.append((ids, offsets))
+        del self._borrowed[:-(self.k_max + 2)]
+
+    def _wrap(self, ptr: int, n_elems: int, dtype: torch.dtype) -> torch.Tensor:
+        off = ptr - self.workspace.data_ptr()
+        nbytes = n_elems * torch.empty((), dtype=dtype).element_size()
+        return self.workspace[off:off + nbytes].view(dtype)
+
+    def out_tensor(self, ptr: int) -> torch.Tensor:
+        return self._wrap(ptr, self.P * self.b * self.T * self.D, torch.float32).view(self.P, self.b, self.T, self.D)
+
+    def __del__(self):
+        h, self.handle = getattr(self, "handle", None), None
+        if h:
+            lib().bls_destroy(h)
+
+
+def bls_plan_bytes(tables: Sequence[torch.Tensor], part: str, P: int, local_batch: int, k_max: int,
+                   max_ids_per_rank: int) -> int:
+    n = C.c_size_t(0)
+    arr = _table_array(tables)
+    _check(lib().bls_plan_bytes(arr, len(tables), PART[part], P, local_batch, k_max,
+                                C.c_int64(max_ids_per_rank), C.byref(n)), "bls_plan_bytes")
+    return n.value
+
+
+def bls_plan(tables: Sequence[torch.Tensor], part: str, P: int, local_batch: int, k_max: int,
+             max_ids_per_rank: int, stream: Optional[torch.cuda.Stream] = None) -> Plan:
+    nbytes = bls_plan_bytes(tables, part, P, local_batch, k_max, max_ids_per_rank)
+    workspace = torch.empty(nbytes + 256, dtype=torch.uint8, device=tables[0].device)
+    pad = (-workspace.data_ptr()) % 256
+    workspace = workspace[pad:pad + nbytes]
+    handle = C.c_void_p()
+    arr = _table_array(tables)
+    _check(lib().bls_plan(arr, len(tables), PART[part], P, local_batch, k_max, C.c_int64(max_ids_per_rank),
+                          C.c_void_p(workspace.data_ptr()), C.c_size_t(nbytes), _stream_ptr(stream),
+                          C.byref(handle)), "bls_plan")
+    return Plan(handle, tables, workspace, P, len(tables), local_batch, tables[0].shape[1], k_max, part, stream)
+
+
+def bls_route(plan: Plan, it: int, ids: torch.Tensor, offsets: torch.Tensor) -> None:
+    plan._keep(ids, offsets)
+    _check(lib().bls_route(plan.handle, C.c_int64(it), C.c_void_p(ids.data_ptr()),
+                           C.c_void_p(offsets.data_ptr()), C.c_int64(ids.numel())), "bls_route")
+
+
+def bls_lookup(plan: Plan, it: int) -> None:
+    _check(lib().bls_lookup(plan.handle, C.c_int64(it)), "bls_lookup")
+
+
+def bls_step(plan: Plan, k: int, ids: torch.Tensor, offsets: torch.Tensor):
+    """Returns (out, out_iter): out is a [P][b][T][D] fp32 view into the ring or None."""
+    plan._keep(ids, offsets)
+    out, it = C.c_void_p(), C.c_int64(-1)
+    _check(lib().bls_step(plan.handle, k, C.c_void_p(ids.data_ptr()), C.c_void_p(offsets.data_ptr()),
+                          C.c_int64(ids.numel()), C.byref(out), C.byref(it)), "bls_step")
+    return (plan.out_tensor(out.value) if out.value else None), it.value
+
+
+def bls_drain(plan: Plan):
+    out, it = C.c_void_p(), C.c_int64(-1)
+    _check(lib().bls_drain(plan.handle, C.byref(out), C.byref(it)), "bls_drain")
+    return (plan.out_tensor(out.value) if out.value else None), it.value
+
+
+def bls_step_host(plan: Plan, k: int, ids: torch.Tensor, offsets: torch.Tensor,
+                  host_out: Optional[torch.Tensor]) -> int:
+    """ids/offsets/host_out are HOST tensors (pinned recommended); returns the iteration copied out or -1."""
+    plan._keep(ids, offsets)
+    it = C.c_int64(-1)
+    _check(lib().bls_step_host(plan.handle, k, C.c_void_p(ids.data_ptr()), C.c_void_p(offsets.data_ptr()),
+                               C.c_int64(ids.numel()),
+                               C.c_void_p(host_out.data_ptr() if host_out is not None else None),
+                               C.byref(it)), "bls_step_host")
+    return it.value
+
+
+def bls_drain_host(plan: Plan, host_out: Optional[torch.Tensor]) -> int:
+    it = C.c_int64(-1)
+    _check(lib().bls_drain_host(plan.handle, C.c_void_p(host_out.data_ptr() if host_out is not None else None),
+                                C.byref(it)), "bls_drain_host")
+    return it.value
+
+
+def bls_view(plan: Plan, it: int) -> dict:
+    """Tensors (views into the ring) of iteration ``it``'s routing artefacts and output."""
+    v = _View()
+    _check(lib().bls_view(plan.handle, C.c_int64(it), C.byref(v)), "bls_view")
+    P = plan.P
+    i32 = torch.int32
+    d = {k: plan._wrap(getattr(v, k), P * P, i32).view(P, P)
+         for k in ("sendcounts", "sdispls", "recvcounts", "rdispls")}
+    d["sendbuf"] = plan._wrap(v.sendbuf, P * v.sendbuf_stride, i32).view(P, v.sendbuf_stride)
+    d["sub_start"] = plan._wrap(v.sub_start, P * v.sub_stride, i32).view(P, v.sub_stride)[:, :v.subbags_per_rank + 1]
+    d["out"] = plan.out_tensor(v.out)
+    return d
+
+
+def bls_counters(plan: Plan):
+    arrs = [(C.c_int64 * plan.P)() for _ in range(3)]
+    _check(lib().bls_counters(plan.handle, *arrs), "bls_counters")
+    return tuple(list(a) for a in arrs)
+
+
+def bls_status(plan: Plan):
+    """(status code, max lag seen); synchronises the plan's stream."""
+    lag = C.c_int64(0)
+    return lib().bls_status(plan.handle, C.byref(lag)), lag.value
+
+
+def bls_set_stall(plan: Plan, rank: int, ns: int) -> None:
+    _check(lib().bls_set_stall(plan.handle, rank, C.c_int64(ns)), "bls_set_stall")
+
+
+def bls_set_wait_limit(plan: Plan, ns: int) -> None:
+    _check(lib().bls_set_wait_limit(plan.handle, C.c_int64(ns)), "bls_set_wait_limit")
+
+
+def bls_fill_hash_table(weight: torch.Tensor, seed: int, t: int,
+                        stream: Optional[torch.cuda.Stream] = None) -> None:
+    _check(lib().bls_fill_hash_table(C.c_void_p(weight.data_ptr()), C.c_int64(weight.shape[0]),
+                                     C.c_int32(weight.shape[1]), _DTYPE[weight.dtype],
+                                     C.c_uint64(seed & ((1 << 64) - 1)), C.c_int32(t), _stream_ptr(stream)),
+           "bls_fill_hash_table")

@@ -1,0 +1,394 @@
+// Host side of the C ABI: workspace layout, plan construction, and the calls
+// that enqueue one wave of kernels (gate -> route -> gather/pool/return -> commit).
+#include <stdio.h>
+#include <stdlib.h>
+#include <string.h>
+#include <vector>
+#include "bls_internal.h"
+
+namespace {
+
+size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+struct Layout {
+    size_t dev, tab, pair, pair_of, counts, sendbuf, sub_start, out, chunk_base, tile_cnt, stage_ids,
+        stage_off, total;
+};
+
+int dtype_bytes(int dt) { return dt == BLS_F32 ? 4 : 2; }
+
+bls_status_t check_shape(const bls_table_t *tables, int T, int part, int P, int b, int k_max,
+                         int64_t cap)
+{
+    if (!tables || T < 1 || P < 1 || P > BLS_MAX_RANKS || b < 1 || k_max < 0 ||
+        k_max + 1 > BLS_MAX_SLOTS || cap < 1 || cap > 0x7fffffff)
+        return BLS_EINVAL;
+    if (part != BLS_PART_TABLE_RR && part != BLS_PART_ROW_BLOCK) return BLS_EINVAL;
+    const int D = tables[0].dim, dt = tables[0].dtype;
+    if (dt != BLS_F32 && dt != BLS_BF16 && dt != BLS_F16) return BLS_EINVAL;
+    const int rb = D * dtype_bytes(dt);
+    if (rb != 16 && rb != 32 && rb != 64 && rb != 128 && rb != 256 && rb != 512) return BLS_EINVAL;
+    for (int t = 0; t < T; t++) {
+        if (tables[t].dim != D || tables[t].dtype != dt) return BLS_EINVAL;
+        if (tables[t].rows < 1 || tables[t].rows > 0x7fffffff) return BLS_EINVAL;
+    }
+    const long long NI = part == BLS_PART_TABLE_RR ? T : (long long)T * P;
+    if (NI * b > 0x7ffffff0LL || (long long)P * T * b > 0x7ffffff0LL) return BLS_EINVAL;
+    return BLS_OK;
+}
+
+void fill_params(BlsParams &p, const bls_table_t *tables, int T, int part, int P, int b, int k_max,
+                 int64_t cap)
+{
+    memset(&p, 0, sizeof(p));
+    p.P = P; p.T = T; p.b = b; p.part = part; p.S = k_max + 1;
+    p.D = tables[0].dim; p.dtype = tables[0].dtype;
+    p.row_bytes = p.D * dtype_bytes(p.dtype);
+    p.lanes = p.row_bytes / 16;
+    p.NI = part == BLS_PART_TABLE_RR ? T : T * P;
+    p.NQ = p.NI * b;
+    p.cap = (int)cap;
+    p.tiles_per_table = (b + BLS_ROUTE_TB - 1) / BLS_ROUTE_TB;
+    p.NT = T * p.tiles_per_table;
+    p.sub_stride = (long long)align_up((size_t)p.NQ + 1, 4);
+    p.out_slot_elems = (long long)P * b * T * p.D;
+}
+
+Layout make_layout(const BlsParams &p)
+{
+    Layout L;
+    size_t o = 0;
+    auto take = [&](size_t bytes) { size_t at = o; o = align_up(o + bytes, 256); return at; };
+    const size_t S = p.S, P = p.P;
+    L.dev = take(sizeof(BlsDev));
+    L.tab = take(sizeof(BlsTableDesc) * p.T);
+    L.pair = take(sizeof(BlsPairDesc) * p.NI);
+    L.pair_of = take(sizeof(int) * p.T);
+    L.counts = take(sizeof(int) * S * 4 * P * P);
+    L.sendbuf = take(sizeof(int) * S * P * (size_t)p.cap);
+    L.sub_start = take(sizeof(int) * S * P * (size_t)p.sub_stride);
+    L.out = take(sizeof(float) * S * (size_t)p.out_slot_elems);
+    L.chunk_base = take(sizeof(int) * P * (size_t)(p.NI + 1));
+    L.tile_cnt = take(p.part == BLS_PART_ROW_BLOCK ? sizeof(int) * P * (size_t)p.NT * P : 0);
+    L.stage_ids = take(sizeof(int) * S * P * (size_t)p.cap);
+    L.stage_off = take(sizeof(int) * S * ((size_t)P * p.T * p.b + 1));
+    L.total = o;
+    return L;
+}
+
+bool cuda_ok(cudaError_t e) { return e == cudaSuccess; }
+
+}  // namespace
+
+extern "C" {
+
+const char *bls_strerror(int s)
+{
+    switch (s) {
+    case BLS_OK: return "ok";
+    case BLS_EINVAL: return "invalid argument or malformed offsets";
+    case BLS_ENOSPC: return "workspace or per-rank ID capacity too small";
+    case BLS_ECUDA: return "CUDA runtime error";
+    case BLS_ERANGE: return "ID out of range";
+    case BLS_ETIMEOUT: return "bounded device-side wait expired";
+    case BLS_ESTATE: return "call order violated or bound out of range";
+    default: return "unknown status";
+    }
+}
+
+bls_status_t bls_plan_bytes(const bls_table_t *tables, int T, int part, int P, int local_batch,
+                            int k_max, int64_t max_ids_per_rank, size_t *bytes)
+{
+    if (!bytes) return BLS_EINVAL;
+    bls_status_t st = check_shape(tables, T, part, P, local_batch, k_max, max_ids_per_rank);
+    if (st != BLS_OK) return st;
+    BlsParams p;
+    fill_params(p, tables, T, part, P, local_batch, k_max, max_ids_per_rank);
+    *bytes = make_layout(p).total;
+    return BLS_OK;
+}
+
+bls_status_t bls_plan(const bls_table_t *tables, int T, int part, int P, int local_batch, int k_max,
+                      int64_t max_ids_per_rank, void *workspace, size_t bytes, void *cuda_stream,
+                      bls_plan_t **plan)
+{
+    if (!plan || !workspace || ((uintptr_t)workspace & 255)) return BLS_EINVAL;
+    bls_status_t st = check_shape(tables, T, part, P, local_batch, k_max, max_ids_per_rank);
+    if (st != BLS_OK) return st;
+    for (int t = 0; t < T; t++)
+        if (!tables[t].weight || ((uintptr_t)tables[t].weight & 15)) return BLS_EINVAL;
+    bls_plan_t *pl = (bls_plan_t *)calloc(1, sizeof(bls_plan_t));
+    if (!pl) return BLS_ENOSPC;
+    BlsParams &p = pl->prm;
+    fill_params(p, tables, T, part, P, local_batch, k_max, max_ids_per_rank);
+    Layout L = make_layout(p);
+    if (bytes < L.total) { free(pl); return BLS_ENOSPC; }
+    char *ws = (char *)workspace;
+    p.dev = (BlsDev *)(ws + L.dev);
+    p.tab = (const BlsTableDesc *)(ws + L.tab);
+    p.pair = (const BlsPairDesc *)(ws + L.pair);
+    p.pair_of_table = (const int *)(ws + L.pair_of);
+    p.counts = (int *)(ws + L.counts);
+    p.sendbuf = (int *)(ws + L.sendbuf);
+    p.sub_start = (int *)(ws + L.sub_start);
+    p.out = (float *)(ws + L.out);
+    p.chunk_base = (int *)(ws + L.chunk_base);
+    p.tile_cnt = (int *)(ws + L.tile_cnt);
+    p.stage_ids = (int *)(ws + L.stage_ids);
+    p.stage_off = (int *)(ws + L.stage_off);
+    pl->stream = (cudaStream_t)cuda_stream;
+    pl->k_max = k_max;
+    pl->k_cur = -1;
+    pl->routed_only = -1;
+    pl->bytes = L.total;
+    int devid = 0;
+    if (!cuda_ok(cudaGetDevice(&devid)) ||
+        !cuda_ok(cudaDeviceGetAttribute(&pl->sm_count, cudaDevAttrMultiProcessorCount, devid))) {
+        free(pl);
+        return BLS_ECUDA;
+    }
+
+    // descriptors
+    std::vector<BlsTableDesc> tab(T);
+    std::vector<BlsPairDesc> pair(p.NI);
+    std::vector<int> pair_of(T, 0);
+    for (int t = 0; t < T; t++) {
+        tab[t].weight = tables[t].weight;
+        tab[t].rows = tables[t].rows;
+        tab[t].blk = part == BLS_PART_ROW_BLOCK ? (int)((tables[t].rows + P - 1) / P) : 0;
+        tab[t].pad = 0;
+    }
+    int n = 0;
+    for (int d = 0; d < P; d++) {
+        for (int t = 0; t < T; t++) {
+            BlsPairDesc q;
+            memset(&q, 0, sizeof(q));
+            q.t = t; q.dst = d;
+            if (part == BLS_PART_TABLE_RR) {
+                if (t % P != d) continue;
+                q.base = tables[t].weight;
+                q.nrows = (int)tables[t].rows;
+                pair_of[t] = n;
+            } else {
+                long long first = (long long)d * tab[t].blk;
+                long long have = tables[t].rows - first;
+                if (have > tab[t].blk) have = tab[t].blk;
+                if (have < 1) { have = 1; first = 0; }      // owner holds nothing: never addressed
+                q.base = (const char *)tables[t].weight + (size_t)first * p.row_bytes;
+                q.nrows = (int)have;
+            }
+            pair[n++] = q;
+        }
+    }
+    BlsDev hd;
+    memset(&hd, 0, sizeof(hd));
+    for (int r = 0; r < BLS_MAX_RANKS; r++) hd.route_iter[r] = hd.serve_iter[r] = hd.consume_iter[r] = -1;
+    hd.wait_limit_ns = 2000000000ull;
+    bool ok = cuda_ok(cudaMemcpyAsync(ws + L.dev, &hd, sizeof(hd), cudaMemcpyHostToDevice, pl->stream)) &&
+              cuda_ok(cudaMemcpyAsync(ws + L.tab, tab.data(), sizeof(BlsTableDesc) * T,
+                                      cudaMemcpyHostToDevice, pl->stream)) &&
+              cuda_ok(cudaMemcpyAsync(ws + L.pair, pair.data(), sizeof(BlsPairDesc) * p.NI,
+                                      cudaMemcpyHostToDevice, pl->stream)) &&
+              cuda_ok(cudaMemcpyAsync(ws + L.pair_of, pair_of.data(), sizeof(int) * T,
+                                      cudaMemcpyHostToDevice, pl->stream)) &&
+              cuda_ok(cudaMemsetAsync(ws + L.counts, 0, sizeof(int) * p.S * 4 * P * P, pl->stream)) &&
+              // the vectors above are pageable: make sure the copies have left them
+              cuda_ok(cudaStreamSynchronize(pl->stream));
+    if (!ok) { free(pl); return BLS_ECUDA; }
+    *plan = pl;
+    return BLS_OK;
+}
+
+void bls_destroy(bls_plan_t *plan) { free(plan); }
+
+static bls_status_t launch_check()
+{
+    return cudaGetLastError() == cudaSuccess ? BLS_OK : BLS_ECUDA;
+}
+
+static const float *slot_out(const bls_plan_t *pl, long long iter)
+{
+    return pl->prm.out + (size_t)(iter % pl->prm.S) * pl->prm.out_slot_elems;
+}
+
+bls_status_t bls_route(bls_plan_t *pl, int64_t iter, const int32_t *ids, const int32_t *offsets,
+                       int64_t n_ids)
+{
+    if (!pl || !offsets || (!ids && n_ids > 0) || n_ids < 0) return BLS_EINVAL;
+    if (iter != pl->t_next || pl->t_handed != pl->t_next || pl->routed_only >= 0) return BLS_ESTATE;
+    bls_launch_gate(pl, BLS_MODE_ROUTE_ONLY, iter, -1, 0, ids, offsets, n_ids);
+    bls_launch_route(pl);
+    bls_launch_commit(pl);
+    pl->routed_only = iter;
+    pl->t_next = iter + 1;
+    return launch_check();
+}
+
+bls_status_t bls_lookup(bls_plan_t *pl, int64_t iter)
+{
+    if (!pl) return BLS_EINVAL;
+    if (pl->routed_only != iter) return BLS_ESTATE;
+    bls_launch_gate(pl, BLS_MODE_LOOKUP_ONLY, iter, -1, 0, nullptr, nullptr, 0);
+    bls_launch_gather(pl);
+    bls_launch_commit(pl);
+    pl->routed_only = -1;
+    pl->t_handed = iter + 1;
+    return launch_check();
+}
+
+bls_status_t bls_step(bls_plan_t *pl, int k, const int32_t *ids, const int32_t *offsets, int64_t n_ids,
+                      const float **out, int64_t *out_iter)
+{
+    if (!pl || !offsets || (!ids && n_ids > 0) || n_ids < 0 || !out || !out_iter) return BLS_EINVAL;
+    if (k < 0 || k > pl->k_max || pl->routed_only >= 0) return BLS_ESTATE;
+    if (pl->k_cur >= 0 && pl->k_cur != k && pl->t_handed != pl->t_next) return BLS_ESTATE;
+    pl->k_cur = k;
+    const long long t = pl->t_next++;
+    bls_launch_gate(pl, BLS_MODE_STEP, t, t - k, k, ids, offsets, n_ids);
+    bls_launch_route(pl);
+    bls_launch_gather(pl);
+    bls_launch_commit(pl);
+    if (t - k >= 0) {
+        *out = slot_out(pl, t - k);
+        *out_iter = t - k;
+        pl->t_handed = t - k + 1;
+    } else {
+        *out = nullptr;
+        *out_iter = -1;
+    }
+    return launch_check();
+}
+
+bls_status_t bls_drain(bls_plan_t *pl, const float **out, int64_t *out_iter)
+{
+    if (!pl || !out || !out_iter) return BLS_EINVAL;
+    if (pl->routed_only >= 0) return BLS_ESTATE;
+    if (pl->t_handed == pl->t_next) {
+        *out = nullptr;
+        *out_iter = -1;
+        pl->k_cur = -1;
+        return BLS_OK;
+    }
+    const long long f = pl->t_handed;
+    bls_launch_gate(pl, BLS_MODE_DRAIN, pl->t_next - 1, f, pl->k_cur < 0 ? 0 : pl->k_cur, nullptr, nullptr, 0);
+    bls_launch_route(pl);
+    bls_launch_gather(pl);
+    bls_launch_commit(pl);
+    *out = slot_out(pl, f);
+    *out_iter = f;
+    pl->t_handed = f + 1;
+    if (pl->t_handed == pl->t_next) pl->k_cur = -1;
+    return launch_check();
+}
+
+bls_status_t bls_step_host(bls_plan_t *pl, int k, const int32_t *ids, const int32_t *offsets,
+                           int64_t n_ids, float *host_out, int64_t *out_iter)
+{
+    if (!pl || !offsets || (!ids && n_ids > 0) || n_ids < 0 || !out_iter) return BLS_EINVAL;
+    const BlsParams &p = pl->prm;
+    if (n_ids > (long long)p.P * p.cap) return BLS_ENOSPC;
+    const int slot = (int)(pl->t_next % p.S);
+    const size_t G1 = (size_t)p.P * p.T * p.b + 1;
+    int *d_ids = p.stage_ids + (size_t)slot * p.P * p.cap;
+    int *d_off = p.stage_off + (size_t)slot * G1;
+    if (cudaMemcpyAsync(d_off, offsets, sizeof(int) * G1, cudaMemcpyHostToDevice, pl->stream) != cudaSuccess ||
+        (n_ids > 0 &&
+         cudaMemcpyAsync(d_ids, ids, sizeof(int) * (size_t)n_ids, cudaMemcpyHostToDevice, pl->stream) != cudaSuccess))
+        return BLS_ECUDA;
+    const float *out = nullptr;
+    bls_status_t st = bls_step(pl, k, d_ids, d_off, n_ids, &out, out_iter);
+    if (st != BLS_OK) return st;
+    if (out && host_out &&
+        cudaMemcpyAsync(host_out, out, sizeof(float) * (size_t)p.out_slot_elems, cudaMemcpyDeviceToHost,
+                        pl->stream) != cudaSuccess)
+        return BLS_ECUDA;
+    return BLS_OK;
+}
+
+bls_status_t bls_drain_host(bls_plan_t *pl, float *host_out, int64_t *out_iter)
+{
+    if (!pl || !out_iter) return BLS_EINVAL;
+    const float *out = nullptr;
+    bls_status_t st = bls_drain(pl, &out, out_iter);
+    if (st != BLS_OK) return st;
+    if (out && host_out &&
+        cudaMemcpyAsync(host_out, out, sizeof(float) * (size_t)pl->prm.out_slot_elems,
+                        cudaMemcpyDeviceToHost, pl->stream) != cudaSuccess)
+        return BLS_ECUDA;
+    return BLS_OK;
+}
+
+bls_status_t bls_view(bls_plan_t *pl, int64_t iter, bls_route_view_t *v)
+{
+    if (!pl || !v) return BLS_EINVAL;
+    if (iter < 0 || iter >= pl->t_next || iter < pl->t_next - pl->prm.S) return BLS_ESTATE;
+    const BlsParams &p = pl->prm;
+    const size_t slot = (size_t)(iter % p.S), PP = (size_t)p.P * p.P;
+    const int *cnt = p.counts + slot * 4 * PP;
+    v->sendcounts = cnt;
+    v->sdispls = cnt + PP;
+    v->recvcounts = cnt + 2 * PP;
+    v->rdispls = cnt + 3 * PP;
+    v->sendbuf = p.sendbuf + slot * p.P * (size_t)p.cap;
+    v->sendbuf_stride = p.cap;
+    v->sub_start = p.sub_start + slot * p.P * (size_t)p.sub_stride;
+    v->sub_stride = p.sub_stride;
+    v->subbags_per_rank = p.NQ;
+    v->out = p.out + slot * (size_t)p.out_slot_elems;
+    return BLS_OK;
+}
+
+bls_status_t bls_counters(bls_plan_t *pl, int64_t *posted, int64_t *served, int64_t *done)
+{
+    if (!pl) return BLS_EINVAL;
+    BlsDev hd;
+    if (cudaStreamSynchronize(pl->stream) != cudaSuccess ||
+        cudaMemcpy(&hd, pl->prm.dev, sizeof(hd), cudaMemcpyDeviceToHost) != cudaSuccess)
+        return BLS_ECUDA;
+    for (int r = 0; r < pl->prm.P; r++) {
+        if (posted) posted[r] = hd.posted[r];
+        if (served) served[r] = hd.served[r];
+        if (done) done[r] = hd.done[r];
+    }
+    return BLS_OK;
+}
+
+bls_status_t bls_status(bls_plan_t *pl, int64_t *max_lag)
+{
+    if (!pl) return BLS_EINVAL;
+    BlsDev hd;
+    if (cudaStreamSynchronize(pl->stream) != cudaSuccess ||
+        cudaMemcpy(&hd, pl->prm.dev, sizeof(hd), cudaMemcpyDeviceToHost) != cudaSuccess)
+        return BLS_ECUDA;
+    if (max_lag) *max_lag = hd.max_lag;
+    if (hd.status & BLS_ST_EINVAL) return BLS_EINVAL;
+    if (hd.status & BLS_ST_ENOSPC) return BLS_ENOSPC;
+    if (hd.status & BLS_ST_ERANGE) return BLS_ERANGE;
+    if (hd.status & BLS_ST_ESTATE) return BLS_ESTATE;
+    if (hd.status & BLS_ST_ETIMEOUT) return BLS_ETIMEOUT;
+    return BLS_OK;
+}
+
+bls_status_t bls_set_stall(bls_plan_t *pl, int rank, int64_t ns)
+{
+    if (!pl || rank < 0 || rank >= pl->prm.P || ns < 0) return BLS_EINVAL;
+    unsigned long long v = (unsigned long long)ns;
+    return cudaMemcpyAsync(&pl->prm.dev->stall_ns[rank], &v, sizeof(v), cudaMemcpyHostToDevice,
+                           pl->stream) == cudaSuccess &&
+                   cudaStreamSynchronize(pl->stream) == cudaSuccess
+               ? BLS_OK
+               : BLS_ECUDA;
+}
+
+bls_status_t bls_set_wait_limit(bls_plan_t *pl, int64_t ns)
+{
+    if (!pl || ns < 0) return BLS_EINVAL;
+    unsigned long long v = (unsigned long long)ns;
+    return cudaMemcpyAsync(&pl->prm.dev->wait_limit_ns, &v, sizeof(v), cudaMemcpyHostToDevice,
+                           pl->stream) == cudaSuccess &&
+                   cudaStreamSynchronize(pl->stream) == cudaSuccess
+               ? BLS_OK
+               : BLS_ECUDA;
+}
+
+}  // extern "C"

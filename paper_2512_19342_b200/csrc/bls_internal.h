@@ -1,0 +1,99 @@
+// Internal structures shared by the kernels and the host API of libbls.
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+#include "bls.h"
+
+#define BLS_MAX_RANKS 32
+#define BLS_MAX_SLOTS 16
+#define BLS_ROUTE_TB 128          // bags per routing tile (row-wise scatter: one thread per bag)
+
+// step modes understood by the gate kernel
+enum { BLS_MODE_STEP = 0, BLS_MODE_DRAIN = 1, BLS_MODE_ROUTE_ONLY = 2, BLS_MODE_LOOKUP_ONLY = 3 };
+
+// bits of the device status word
+enum { BLS_ST_EINVAL = 1, BLS_ST_ENOSPC = 2, BLS_ST_ERANGE = 4, BLS_ST_ETIMEOUT = 8, BLS_ST_ESTATE = 16 };
+
+// Device-resident state of the slot ring.  Counters are monotone: posted[r] =
+// iterations whose requests rank r has put into the owners' slots, served[o] =
+// iterations owner o has answered, done[r] = iterations rank r has completed.
+struct BlsDev {
+    long long posted[BLS_MAX_RANKS];
+    long long served[BLS_MAX_RANKS];
+    long long done[BLS_MAX_RANKS];
+    unsigned long long ready_ns[BLS_MAX_RANKS];   // rank may act again at this globaltimer value
+    unsigned long long stall_ns[BLS_MAX_RANKS];   // injected delay before each iteration
+    // plan of the current wave: iteration each rank routes / serves / completes, or -1
+    long long route_iter[BLS_MAX_RANKS];
+    long long serve_iter[BLS_MAX_RANKS];
+    long long consume_iter[BLS_MAX_RANKS];
+    // inputs of the iterations that are still in the ring, by slot
+    const int *in_ids[BLS_MAX_SLOTS];
+    const int *in_off[BLS_MAX_SLOTS];
+    long long in_n[BLS_MAX_SLOTS];
+    unsigned long long wait_limit_ns;
+    long long max_lag;                            // max over time of newest posted - oldest incomplete
+    int status;                                   // OR of BLS_ST_* bits
+    int pad;
+};
+
+struct BlsTableDesc {
+    const void *weight;
+    long long rows;
+    int blk;            // ceil(rows / P) for row-block placement, else 0
+    int pad;
+};
+
+// A (owner, table) pair in owner-major order.  Table-wise: one pair per table.
+// Row-wise: P pairs per table.
+struct BlsPairDesc {
+    const void *base;   // first row this owner holds of the table
+    int t;              // table number
+    int dst;            // owner rank
+    int nrows;          // rows the owner holds (for clamping); >= 1
+    int pad;
+};
+
+struct BlsParams {
+    int P, T, b, part, S, D, dtype, lanes;
+    int NI;                 // number of (owner, table) pairs
+    int NQ;                 // sub-bags per requester = NI * b
+    int cap;                // IDs per rank per iteration (send buffer capacity)
+    int NT;                 // routing tiles per requester = T * ceil(b / TB)
+    int tiles_per_table;    // ceil(b / TB)
+    int row_bytes;
+    BlsDev *dev;
+    const BlsTableDesc *tab;     // [T]
+    const BlsPairDesc *pair;     // [NI]
+    const int *pair_of_table;    // [T] index of table t's (first) pair; row-wise: unused
+    int *counts;                 // [S][4][P][P]: sendcounts, sdispls, recvcounts, rdispls
+    int *sendbuf;                // [S][P][cap]
+    int *sub_start;              // [S][P][sub_stride]
+    float *out;                  // [S][P][b][T][D]
+    int *chunk_base;             // [P][NI+1]   table-wise: start of each (src, table) chunk
+    int *tile_cnt;               // [P][NT][P]  row-wise: per tile, per destination counts / bases
+    int *stage_ids;              // [S][P*cap]  staging for host inputs
+    int *stage_off;              // [S][G+1]
+    long long sub_stride;        // NQ + 1 rounded up to a multiple of 4
+    long long out_slot_elems;    // P*b*T*D
+};
+
+struct bls_plan {
+    BlsParams prm;
+    cudaStream_t stream;
+    int k_max;
+    int k_cur;              // bound in use, -1 when nothing is outstanding
+    long long t_next;       // next iteration to issue
+    long long t_handed;     // iterations handed back so far
+    long long routed_only;  // iteration routed by bls_route and not yet looked up, or -1
+    size_t bytes;
+    int sm_count;
+};
+
+// kernel launchers (defined in the .cu files)
+void bls_launch_gate(const bls_plan_t *pl, int mode, long long t_last, long long forced_floor, int k,
+                     const int *ids, const int *off, long long n_ids);
+void bls_launch_commit(const bls_plan_t *pl);
+void bls_launch_route(const bls_plan_t *pl);
+void bls_launch_gather(const bls_plan_t *pl);
+void bls_launch_init(const bls_plan_t *pl, const BlsDev *host_dev);

@@ -1,0 +1,168 @@
+// Slot ring of the bounded-lag-synchronous exchange: per-rank progress counters
+// in device memory, the gate that decides what every logical rank may do in the
+// next wave of kernels, and the commit that publishes the wave's progress.
+//
+// Reading of the paper (Section III-C, III-D, Section IV / Listing 2):
+//   * iteration j uses slot j mod S, S = k_max + 1 buffers created at plan time;
+//   * a rank may put the requests of iteration j only when every rank has
+//     completed iteration j - k - 1, i.e. min(done) >= j - k (otherwise it
+//     "will overwrite buffer", Listing 2);
+//   * an owner answers iteration j once all P sources have posted it (tagged
+//     messages are counted per iteration);
+//   * a rank completes iteration j once all owners have answered it; completion
+//     is oldest first; the oldest request must complete once more than k are
+//     outstanding; the last batch drains everything.
+// A rank under an injected delay takes no action until its delay has passed,
+// unless the bound forces it; then the gate waits (bounded) on the clock.
+#include "bls_internal.h"
+
+__device__ __forceinline__ unsigned long long globaltimer_ns()
+{
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+
+__device__ __forceinline__ long long warp_min_ll(long long v)
+{
+    for (int o = 16; o > 0; o >>= 1) {
+        long long w = __shfl_xor_sync(0xffffffffu, v, o);
+        v = w < v ? w : v;
+    }
+    return v;
+}
+__device__ __forceinline__ long long warp_max_ll(long long v)
+{
+    for (int o = 16; o > 0; o >>= 1) {
+        long long w = __shfl_xor_sync(0xffffffffu, v, o);
+        v = w > v ? w : v;
+    }
+    return v;
+}
+
+// One warp; lane r is logical rank r.
+__global__ void __launch_bounds__(32) bls_gate_kernel(BlsParams p, int mode, long long t_last,
+                                                      long long floor_, int k, const int *ids,
+                                                      const int *off, long long n_ids)
+{
+    BlsDev *d = p.dev;
+    const int r = threadIdx.x;
+    const bool act = r < p.P;
+    const long long BIG = 0x7fffffffffffffffLL;
+
+    if (r == 0 && (mode == BLS_MODE_STEP || mode == BLS_MODE_ROUTE_ONLY)) {
+        int slot = (int)(t_last % p.S);
+        d->in_ids[slot] = ids;
+        d->in_off[slot] = off;
+        d->in_n[slot] = n_ids;
+    }
+    __syncwarp();
+
+    long long posted = act ? d->posted[r] : BIG;
+    long long served = act ? d->served[r] : BIG;
+    long long done = act ? d->done[r] : BIG;
+    unsigned long long ready_at = act ? d->ready_ns[r] : 0ull;
+    const bool sync_mode = (mode == BLS_MODE_ROUTE_ONLY || mode == BLS_MODE_LOOKUP_ONLY);
+
+    // Ranks the bound forces to act in this wave: anything still at or below the floor.
+    bool forced = act && (sync_mode || (floor_ >= 0 && (posted <= floor_ || served <= floor_ || done <= floor_)));
+
+    // Bounded wait on the clock for the forced ranks' injected delays.
+    unsigned long long need = forced ? ready_at : 0ull;
+    for (int o = 16; o > 0; o >>= 1) {
+        unsigned long long w = __shfl_xor_sync(0xffffffffu, need, o);
+        need = w > need ? w : need;
+    }
+    unsigned long long now = globaltimer_ns();
+    if (!sync_mode && need > now) {
+        const unsigned long long give_up = now + d->wait_limit_ns;
+        while (now < need && now < give_up) {
+            __nanosleep(1000);
+            now = globaltimer_ns();
+        }
+        if (now < need && r == 0) atomicOr(&d->status, BLS_ST_ETIMEOUT);
+    }
+    const bool is_ready = forced || now >= ready_at;
+
+    const long long min_done = warp_min_ll(done);
+
+    // post: slot of iteration `posted` is free once every rank completed posted - k - 1
+    bool go_r = act && mode != BLS_MODE_LOOKUP_ONLY && posted <= t_last &&
+                min_done >= posted - k && is_ready;
+    long long posted2 = act ? posted + (go_r ? 1 : 0) : BIG;
+    const long long min_posted2 = warp_min_ll(posted2);
+    const long long max_posted2 = warp_max_ll(act ? posted2 : -1);
+
+    // serve: all P sources (self included) have posted the iteration
+    bool go_s = act && mode != BLS_MODE_ROUTE_ONLY && served < min_posted2 && is_ready;
+    long long served2 = act ? served + (go_s ? 1 : 0) : BIG;
+    const long long min_served2 = warp_min_ll(served2);
+
+    // complete: all owners have answered; oldest first
+    bool go_c = act && mode != BLS_MODE_ROUTE_ONLY && done < min_served2 && is_ready;
+    long long done2 = act ? done + (go_c ? 1 : 0) : BIG;
+    const long long min_done2 = warp_min_ll(done2);
+
+    if (act) {
+        d->route_iter[r] = go_r ? posted : -1;
+        d->serve_iter[r] = go_s ? served : -1;
+        d->consume_iter[r] = go_c ? done : -1;
+    }
+    if (r == 0) {
+        long long lag = max_posted2 - 1 - min_done;
+        if (lag > d->max_lag) d->max_lag = lag;
+        // the wave must satisfy the bound: everything up to the floor completes
+        if (!sync_mode && floor_ >= 0 && min_done2 <= floor_) atomicOr(&d->status, BLS_ST_ESTATE);
+        if (mode == BLS_MODE_ROUTE_ONLY && min_posted2 <= t_last) atomicOr(&d->status, BLS_ST_ESTATE);
+        if (mode == BLS_MODE_LOOKUP_ONLY && min_done2 <= t_last) atomicOr(&d->status, BLS_ST_ESTATE);
+    }
+}
+
+// One warp; publishes the progress of the wave that has just run and starts the
+// injected delay of every rank that posted.  For every answered iteration it
+// also writes the receive-side counts and displacements of the request leg
+// (recvcounts = sendcounts transposed, rdispls = exclusive scan over sources).
+__global__ void __launch_bounds__(32) bls_commit_kernel(BlsParams p)
+{
+    BlsDev *d = p.dev;
+    const int r = threadIdx.x;
+    if (r >= p.P) return;
+    const unsigned long long now = globaltimer_ns();
+    long long j = d->route_iter[r];
+    if (j >= 0) {
+        d->posted[r] = j + 1;
+        d->ready_ns[r] = now + d->stall_ns[r];
+        d->route_iter[r] = -1;
+    }
+    j = d->serve_iter[r];
+    if (j >= 0) {
+        int *cnt = p.counts + (size_t)(j % p.S) * 4 * p.P * p.P;
+        const int *sendcounts = cnt;
+        int *recvcounts = cnt + 2 * p.P * p.P, *rdispls = cnt + 3 * p.P * p.P;
+        int run = 0;
+        for (int src = 0; src < p.P; src++) {
+            int c = sendcounts[src * p.P + r];
+            recvcounts[r * p.P + src] = c;
+            rdispls[r * p.P + src] = run;
+            run += c;
+        }
+        d->served[r] = j + 1;
+        d->serve_iter[r] = -1;
+    }
+    j = d->consume_iter[r];
+    if (j >= 0) {
+        d->done[r] = j + 1;
+        d->consume_iter[r] = -1;
+    }
+}
+
+void bls_launch_gate(const bls_plan_t *pl, int mode, long long t_last, long long forced_floor, int k,
+                     const int *ids, const int *off, long long n_ids)
+{
+    bls_gate_kernel<<<1, 32, 0, pl->stream>>>(pl->prm, mode, t_last, forced_floor, k, ids, off, n_ids);
+}
+
+void bls_launch_commit(const bls_plan_t *pl)
+{
+    bls_commit_kernel<<<1, 32, 0, pl->stream>>>(pl->prm);
+}

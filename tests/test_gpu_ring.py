@@ -1,0 +1,156 @@
+"""The BLS slot ring on the GPU: output for any bound k equals the synchronous
+output (Abstract: accuracy is fully preserved; Section III-D: k = 0 is the plain
+alltoallv), ranks really lag under injected delays, never by more than k, and a
+wait that cannot end in time returns a status instead of hanging.  GPU only."""
+import numpy as np
+import pytest
+import torch
+
+import bls_inputs as bi
+import oracle
+import paper_2512_19342_b200 as bls
+from test_gpu_parity import TOL, check_route, dev_tables, make_plan
+
+pytestmark = pytest.mark.gpu
+
+
+def run_loop(w, tabs, k, n_iter, k_max=None, stalls=None, check_views=False, wait_limit=None):
+    """Listing 2's loop: n_iter steps then the drain; returns {iteration: output}."""
+    plan = make_plan(w, tabs, k if k_max is None else k_max)
+    if wait_limit is not None:
+        bls.bls_set_wait_limit(plan, wait_limit)
+    for r, ns in (stalls or {}).items():
+        bls.bls_set_stall(plan, r, ns)
+    outs, inputs = {}, []
+    for t in range(n_iter):
+        ids, off = bi.make_iteration(w, t)
+        inputs.append((ids, off))
+        d_ids, d_off = torch.from_numpy(ids).cuda(), torch.from_numpy(off).cuda()
+        out, it = bls.bls_step(plan, k, d_ids, d_off)
+        if t < k:
+            assert out is None and it == -1
+        else:
+            assert it == t - k
+            outs[it] = out.clone()
+        if check_views and not stalls:
+            check_route(w, bls.bls_view(plan, t), ids, off)
+    while True:
+        out, it = bls.bls_drain(plan)
+        if out is None:
+            break
+        assert it == len(outs)                    # oldest first
+        outs[it] = out.clone()
+    status, lag = bls.bls_status(plan)
+    posted, served, done = bls.bls_counters(plan)
+    assert posted == served == done == [n_iter] * w.P
+    return outs, inputs, status, lag
+
+
+@pytest.mark.parametrize("num,rs,bs", [(1, 1.0, 1.0), (3, 0.01, 0.02), (4, 0.002, 0.01)])
+def test_output_is_independent_of_k(num, rs, bs):
+    w = bi.workload(num, rs, bs)
+    data = [bi.table_values(t) for t in w.tables]
+    tabs = dev_tables(w, data)
+    n_iter = 7
+    ref, inputs, status, lag = run_loop(w, tabs, 0, n_iter, check_views=True)
+    assert status == bls.BLS_OK and lag == 0 and sorted(ref) == list(range(n_iter))
+    P, T, b = w.P, w.T, w.local_batch
+    for it, (ids, off) in enumerate(inputs):
+        want = oracle.pool_definition(P, T, b, w.tables, data, ids, off)
+        assert oracle.vector_rel_err(ref[it].cpu().numpy(), want) <= TOL[w.tables[0].dtype]
+    for k in (1, 2, 4, 8):
+        outs, _, status, lag = run_loop(w, tabs, k, n_iter, check_views=True)
+        assert status == bls.BLS_OK and lag <= k
+        assert sorted(outs) == list(range(n_iter))
+        for it in range(n_iter):
+            if w.partition == "table_rr":
+                assert torch.equal(outs[it], ref[it]), (k, it)       # deterministic kernels: bit-identical
+            else:                                                     # partial sums are added in arrival order
+                assert oracle.vector_rel_err(outs[it].cpu().numpy(), ref[it].cpu().numpy()) <= 1e-5
+
+
+def test_ring_larger_than_bound():
+    """A plan made for k_max = 4 also serves k = 1 (fewer slots in flight)."""
+    w = bi.workload(1)
+    tabs = dev_tables(w, [bi.table_values(t) for t in w.tables])
+    ref, *_ = run_loop(w, tabs, 0, 5)
+    outs, _, status, _ = run_loop(w, tabs, 1, 5, k_max=4)
+    assert status == bls.BLS_OK
+    assert all(torch.equal(outs[i], ref[i]) for i in range(5))
+
+
+@pytest.mark.parametrize("part", ["table_rr", "row_block"])
+def test_delayed_ranks_lag_within_the_bound(part):
+    """Injected delays (Section V-E, setting 2) make ranks fall behind; the
+    counters keep them within k iterations and the results do not change."""
+    w = bi.tiny_workload(T=4, P=4, b=64, rows=500, dim=16, partition=part, lengths="poisson10")
+    data = [bi.table_values(t) for t in w.tables]
+    tabs = dev_tables(w, data)
+    n_iter = 10
+    ref, *_ = run_loop(w, tabs, 0, n_iter)
+    for k in (1, 3):
+        outs, _, status, lag = run_loop(w, tabs, k, n_iter, stalls={1: 3_000_000, 2: 500_000})
+        assert status == bls.BLS_OK
+        assert 1 <= lag <= k, lag                                     # somebody really ran ahead
+        for it in range(n_iter):
+            assert oracle.vector_rel_err(outs[it].cpu().numpy(), ref[it].cpu().numpy()) <= 1e-5
+    # bound 0: the delay is paid every iteration, nobody runs ahead
+    outs, _, status, lag = run_loop(w, tabs, 0, 4, stalls={1: 1_000_000})
+    assert status == bls.BLS_OK and lag == 0
+    assert all(torch.equal(outs[i], ref[i]) or part == "row_block" for i in range(4))
+
+
+def test_wait_that_cannot_end_returns_a_status():
+    """A delay longer than the wait limit: the gate gives up, records
+    BLS_ETIMEOUT, goes on with correct data, and the context stays usable."""
+    w = bi.workload(1)
+    tabs = dev_tables(w, [bi.table_values(t) for t in w.tables])
+    ref, *_ = run_loop(w, tabs, 0, 3)
+    outs, _, status, _ = run_loop(w, tabs, 0, 3, stalls={0: 5_000_000_000}, wait_limit=200_000)
+    assert status == bls.BLS_ETIMEOUT
+    assert all(torch.equal(outs[i], ref[i]) for i in range(3))
+    assert torch.ones(8, device="cuda").sum().item() == 8.0
+
+
+def test_changing_k_mid_flight_is_refused():
+    w = bi.workload(1)
+    tabs = dev_tables(w, [bi.table_values(t) for t in w.tables])
+    plan = make_plan(w, tabs, 2)
+    ids, off = bi.make_iteration(w, 0)
+    d_ids, d_off = torch.from_numpy(ids).cuda(), torch.from_numpy(off).cuda()
+    bls.bls_step(plan, 2, d_ids, d_off)
+    with pytest.raises(bls.BlsError) as e:
+        bls.bls_step(plan, 1, d_ids, d_off)
+    assert e.value.code == bls.BLS_ESTATE
+    while bls.bls_drain(plan)[0] is not None:
+        pass
+    out, it = bls.bls_step(plan, 0, d_ids, d_off)              # allowed again after the drain
+    assert it == 1 and out is not None
+
+
+def test_host_buffer_entry_points():
+    """bls_step_host / bls_drain_host: host IDs in, host vectors out."""
+    w = bi.workload(3, 0.01, 0.02)
+    data = [bi.table_values(t) for t in w.tables]
+    tabs = dev_tables(w, data)
+    plan = make_plan(w, tabs, 1)
+    P, T, b, D = w.P, w.T, w.local_batch, w.tables[0].dim
+    host_out = torch.empty(P, b, T, D, dtype=torch.float32).pin_memory()
+    got, inputs = {}, []
+    for t in range(4):
+        ids, off = bi.make_iteration(w, t)
+        inputs.append((ids, off))
+        it = bls.bls_step_host(plan, 1, torch.from_numpy(ids).pin_memory(), torch.from_numpy(off).pin_memory(), host_out)
+        torch.cuda.synchronize()
+        if it >= 0:
+            got[it] = host_out.clone()
+    while True:
+        it = bls.bls_drain_host(plan, host_out)
+        torch.cuda.synchronize()
+        if it < 0:
+            break
+        got[it] = host_out.clone()
+    assert sorted(got) == [0, 1, 2, 3] and bls.bls_status(plan)[0] == bls.BLS_OK
+    for it, (ids, off) in enumerate(inputs):
+        want = oracle.pool_definition(P, T, b, w.tables, data, ids, off)
+        assert oracle.vector_rel_err(got[it].numpy(), want) <= 1e-5
