@@ -1,0 +1,425 @@
+#!/usr/bin/env python
+"""Benchmark of the BLS embedding-lookup hot path.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--config C] [--impl reference]
+
+A step is one pass of the whole hot path (route -> gather/pool -> return, inside
+the slot ring) over one batch of synthetic input.  Prints ONE JSON line.
+With N > 1 (torchrun) every rank runs an independent replica of the workload
+(the path has no exchange between GPUs); the value is the sum over replicas
+divided by the slowest replica's device time.
+"""
+from __future__ import annotations
+
+import argparse
+import hashlib
+import json
+import os
+import statistics
+import subprocess
+import sys
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import bls_inputs as bi  # noqa: E402
+
+NOMINAL_HBM_GBS = 8000.0
+FALLBACK_HBM_GBS = 6650.0
+DT_BYTES = {"f32": 4, "bf16": 2, "f16": 2}
+N_DISTINCT = {1: 10, 2: 16, 3: 8, 4: 3, 5: 3}       # distinct ID batches kept resident and cycled
+
+
+def parse_args():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=300)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--config", type=int, default=3, help="workload 1..5 (3 = 26-table Zipf multi-hot)")
+    ap.add_argument("--impl", default="mine", choices=["mine", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--tables", type=int, default=0, help="keep only the first N tables (reduced profiling case)")
+    ap.add_argument("--ks", default="", help="comma-separated bounds to time instead of the workload's own")
+    return ap.parse_args()
+
+
+def dist_env():
+    return int(os.environ.get("RANK", 0)), int(os.environ.get("LOCAL_RANK", 0)), int(os.environ.get("WORLD_SIZE", 1))
+
+
+def measured_peak():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        try:
+            return float(json.load(open(path))["hbm_gbs"]), "measured"
+        except Exception:
+            pass
+    return FALLBACK_HBM_GBS, "fallback"
+
+
+def algorithmic_bytes(w, L: int):
+    """Bytes the method itself must move per iteration.
+
+    whole step: rows (every lookup, duplicates included) + IDs three times (read,
+    write packed, read packed) + bag boundaries three times + output once.
+    gather kernel alone: rows + packed IDs once + sub-bag starts once + output once.
+    """
+    r = w.tables[0].dim * DT_BYTES[w.tables[0].dtype]
+    G = w.n_bags
+    Gp = G if w.partition == "table_rr" else G * w.P
+    out = G * w.tables[0].dim * 4
+    step = L * r + 3 * L * 4 + 3 * Gp * 4 + out
+    gather = L * r + L * 4 + Gp * 4 + out
+    return step, gather
+
+
+class ClockSampler:
+    """nvidia-smi clock / throttle-reason samples taken while the timed loops run."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.path = f"/tmp/bls_clocks_{os.getpid()}.csv"
+        self.proc = None
+        try:
+            self.fh = open(self.path, "w")
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                                          "-lms", "50", "-i", str(index)], stdout=self.fh, stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        self.fh.close()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in open(self.path):
+            f = [x.strip() for x in line.split(",")]
+            if len(f) < 7:
+                continue
+            try:
+                sm.append(float(f[0]))
+                mx.append(float(f[1]))
+            except ValueError:
+                continue
+            for n, v in zip(names, f[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        try:
+            os.remove(self.path)
+        except OSError:
+            pass
+        # the box idles between launches of this short benchmark: report the upper half as "under load"
+        load = sorted(sm)[len(sm) // 2:] if sm else []
+        return {"sm_mhz": statistics.median(load) if load else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+def host_inputs(w, n_distinct):
+    return [bi.make_iteration(w, it) for it in range(n_distinct)]
+
+
+def capacity(w, inputs):
+    tb = w.T * w.local_batch
+    return max(int(np.diff(off[::tb].astype(np.int64)).max()) for _, off in inputs) + 64
+
+
+def traffic_record(kernel_src: str, workload_name: str):
+    """DRAM bytes per launch of the gather kernel from the committed ncu capture,
+    or None when the kernel source has changed since the counters were taken."""
+    path = os.path.join(ROOT, "profiles", "gather_pool_traffic.json")
+    if not os.path.exists(path):
+        return None
+    try:
+        rec = json.load(open(path))
+        digest = hashlib.sha256(open(kernel_src, "rb").read()).hexdigest()
+        if rec.get("kernel_sha256") != digest or rec.get("workload") != workload_name:
+            return None
+        return float(rec["dram_bytes_per_launch"])
+    except Exception:
+        return None
+
+
+# --------------------------------------------------------------------------
+# CPU oracle legs (the only places this program executes anything under oracle/)
+# --------------------------------------------------------------------------
+def host_tables_for_oracle(w, cores):
+    """Materialise the tables on the host when they fit comfortably, else evaluate rows on demand."""
+    import oracle
+    need = w.table_bytes()
+    avail = 0
+    try:
+        for line in open("/proc/meminfo"):
+            if line.startswith("MemAvailable"):
+                avail = int(line.split()[1]) * 1024
+    except OSError:
+        pass
+    if need * 3 > avail:
+        return None, "rows evaluated on demand from the counter hash"
+    data = []
+    for spec in w.tables:
+        data.append(oracle.fill_table(spec, nthreads=cores) if spec.kind == "hash" else bi.table_values(spec))
+    return data, "tables materialised in host memory"
+
+
+def oracle_iteration(w, data, ids, off, cores):
+    import oracle
+    oracle.route(w.P, w.T, w.local_batch, w.partition, [t.rows for t in w.tables], ids, off, nthreads=cores)
+    oracle.pool_definition(w.P, w.T, w.local_batch, w.tables, data, ids, off, nthreads=cores)
+
+
+def cpu_baseline(w, inputs, target_s=12.0):
+    cores = len(os.sched_getaffinity(0))
+    data, how = host_tables_for_oracle(w, cores)
+    ids, off = inputs[0]
+    t0 = time.perf_counter()
+    oracle_iteration(w, data, ids, off, cores)
+    t1 = time.perf_counter() - t0
+    n = int(max(1, min(len(inputs) * 4, round(target_s / max(t1, 1e-3)))))
+    lookups = 0
+    t0 = time.perf_counter()
+    for i in range(n):
+        ids, off = inputs[i % len(inputs)]
+        oracle_iteration(w, data, ids, off, cores)
+        lookups += len(ids)
+    dt = time.perf_counter() - t0
+    return {"value": lookups / dt, "unit": "lookups/s", "cores": cores, "kind": "oracle",
+            "sample": f"{n} full iteration(s) of {w.name} ({lookups} lookups, {dt:.1f} s): route + fp64 pooling by "
+                      f"definition, one OpenMP thread per core; {how}"}
+
+
+def run_reference(args):
+    """--impl reference: the oracle, as it stands, timed on the host cores."""
+    rank, _, world = dist_env()
+    if rank != 0:
+        return
+    cores = len(os.sched_getaffinity(0))
+    w_full = bi.workload(args.config)
+    data, how = host_tables_for_oracle(w_full, cores)
+    probe_scale = 1.0 / 16
+    wp = bi.workload(args.config, 1.0, probe_scale)
+    ids, off = bi.make_iteration(wp, 0)
+    t0 = time.perf_counter()
+    oracle_iteration(wp, data, ids, off, cores)
+    t_probe = time.perf_counter() - t0
+    budget = 120.0 / max(1, args.steps + args.warmup)
+    scale = min(1.0, probe_scale * budget / max(t_probe, 1e-4))
+    ws = bi.workload(args.config, 1.0, scale)
+    inputs = host_inputs(ws, min(4, N_DISTINCT[args.config]))
+    for i in range(args.warmup):
+        oracle_iteration(ws, data, *inputs[i % len(inputs)], cores)
+    lookups = 0
+    t0 = time.perf_counter()
+    for i in range(args.steps):
+        ids, off = inputs[i % len(inputs)]
+        oracle_iteration(ws, data, ids, off, cores)
+        lookups += len(ids)
+    dt = time.perf_counter() - t0
+    val = lookups / dt
+    sample = (f"each step = one iteration of {w_full.name} at global batch {ws.global_batch} of "
+              f"{w_full.global_batch} ({lookups // max(1, args.steps)} lookups/step); {how}")
+    print(json.dumps({
+        "impl": "reference", "metric": "embedding_lookups_per_s", "value": val, "unit": "lookups/s",
+        "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt / args.steps * 1e3,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": w_full.tables[0].dtype,
+        "data": "synthetic", "config": {"workload": w_full.name, "P": w_full.P, "partition": w_full.partition,
+                                        "global_batch": ws.global_batch, "sample": sample},
+        "cpu_baseline": {"value": val, "unit": "lookups/s", "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": val, "unit": "lookups/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }))
+
+
+# --------------------------------------------------------------------------
+# the CUDA path
+# --------------------------------------------------------------------------
+def aggregate(elapsed_ms: float, units: float, world: int, device=None):
+    """Whole-job figure: units summed over ranks, time = max over ranks."""
+    if world == 1:
+        return elapsed_ms, units
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([elapsed_ms], dtype=torch.float64, device=device)
+    u = torch.tensor([units], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    dist.all_reduce(u, op=dist.ReduceOp.SUM)
+    return float(t.item()), float(u.item())
+
+
+def device_tables(w, bls, torch):
+    tdt = {"f32": torch.float32, "bf16": torch.bfloat16, "f16": torch.float16}
+    tabs = []
+    for spec in w.tables:
+        if spec.kind == "hash":
+            t = torch.empty(spec.rows, spec.dim, dtype=tdt[spec.dtype], device="cuda")
+            bls.bls_fill_hash_table(t, spec.seed, spec.index)
+        else:
+            v = bi.table_values(spec)
+            t = torch.from_numpy(v.view(np.int16) if spec.dtype == "bf16" else v)
+            t = (t.view(torch.bfloat16) if spec.dtype == "bf16" else t).cuda()
+        tabs.append(t)
+    torch.cuda.synchronize()
+    return tabs
+
+
+def select(w, args):
+    """Optional reductions of the workload for profiling runs."""
+    import dataclasses
+    if args.tables:
+        w = dataclasses.replace(w, tables=w.tables[:args.tables], name=f"{w.name}_first{args.tables}tables")
+    if args.ks:
+        w = dataclasses.replace(w, ks=tuple(int(x) for x in args.ks.split(",")))
+    return w
+
+
+def run_mine(args):
+    import torch
+    import paper_2512_19342_b200 as bls
+    rank, local_rank, world = dist_env()
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+
+    def barrier():
+        if world > 1:
+            import torch.distributed as dist
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    w = select(bi.workload(args.config), args)
+    nd = N_DISTINCT[args.config]
+    inputs = host_inputs(w, nd)
+    tabs = device_tables(w, bls, torch)
+    d_in = [(torch.from_numpy(i).cuda(), torch.from_numpy(o).cuda()) for i, o in inputs]
+    Ls = [len(i) for i, _ in inputs]
+    k_max = max(w.ks)
+    plan = bls.bls_plan(tabs, w.partition, w.P, w.local_batch, k_max, capacity(w, inputs))
+
+    def loop(k, steps):
+        for t in range(steps):
+            ids, off = d_in[t % nd]
+            bls.bls_step(plan, k, ids, off)
+        while bls.bls_drain(plan)[0] is not None:
+            pass
+
+    def timed(k, steps):
+        barrier()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        loop(k, steps)
+        e1.record()
+        barrier()
+        return e0.elapsed_time(e1)
+
+    ks = sorted(set(w.ks) | {0})
+    k_head = max(w.ks)
+    loop(k_head, max(3, args.warmup))
+    torch.cuda.synchronize()
+    st, _ = bls.bls_status(plan)
+    if st != bls.BLS_OK:
+        raise RuntimeError(f"device status {st} after warm-up")
+
+    sampler = ClockSampler(local_rank) if rank == 0 else None
+    units = float(sum(Ls[t % nd] for t in range(args.steps)))
+    by_k = {}
+    launches = 0
+    for k in ks:
+        n0 = bls.bls_profile_read(plan)["kernels_total"]
+        ms, tot = aggregate(timed(k, args.steps), units, world, dev)
+        by_k[k] = (ms, tot)
+        if k == k_head:
+            launches = bls.bls_profile_read(plan)["kernels_total"] - n0   # counted by the library
+    # stage times of the same loop (k = 0: every call runs every stage), CUDA events on the plan's stream
+    bls.bls_profile(plan, True)
+    loop(0, min(args.steps, 1000))
+    prof = bls.bls_profile_read(plan)
+    bls.bls_profile(plan, False)
+    # end to end through the host-buffer entry points
+    e2e = None
+    if not args.no_e2e:
+        h_in = [(torch.from_numpy(i).pin_memory(), torch.from_numpy(o).pin_memory()) for i, o in inputs]
+        h_out = torch.empty(w.P, w.local_batch, w.T, w.tables[0].dim, dtype=torch.float32).pin_memory()
+        n_e2e = max(3, min(args.steps, 100))
+
+        def loop_host(steps):
+            for t in range(steps):
+                bls.bls_step_host(plan, k_head, h_in[t % nd][0], h_in[t % nd][1], h_out)
+            while bls.bls_drain_host(plan, h_out) >= 0:
+                pass
+        loop_host(3)
+        barrier()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        loop_host(n_e2e)
+        e1.record()
+        barrier()
+        u_e = float(sum(Ls[t % nd] for t in range(n_e2e)))
+        ms_e, tot_e = aggregate(e0.elapsed_time(e1), u_e, world, dev)
+        e2e = {"value": tot_e / (ms_e * 1e-3), "unit": "lookups/s",
+               "h2d_bytes_per_step": int(np.mean([i.nbytes + o.nbytes for i, o in inputs])),
+               "d2h_bytes_per_step": int(h_out.numel() * 4), "steps": n_e2e, "k": k_head}
+    clocks = sampler.stop() if sampler else None
+    st, lag = bls.bls_status(plan)
+    if st != bls.BLS_OK:
+        raise RuntimeError(f"device status {st} after the timed loops")
+    if rank != 0:
+        return
+
+    ms_head, tot_head = by_k[k_head]
+    peak, peak_src = measured_peak()
+    L_mean = float(np.mean(Ls))
+    step_bytes, gather_bytes = algorithmic_bytes(w, L_mean)
+    ms_gather = prof["ms_gather"] / max(1, prof["calls"])
+    ach = gather_bytes / (ms_gather * 1e-3) / 1e9
+    step_gbs = step_bytes * world / (ms_head / args.steps * 1e-3) / 1e9
+    result = {
+        "metric": "embedding_lookups_per_s", "value": tot_head / (ms_head * 1e-3), "unit": "lookups/s",
+        "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_head / args.steps,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": w.tables[0].dtype,
+        "data": "synthetic",
+        "config": {"workload": w.name, "tables": w.T, "rows": [t.rows for t in w.tables][:3] + ["..."],
+                   "dim": w.tables[0].dim, "P": w.P, "partition": w.partition, "global_batch": w.global_batch,
+                   "lookups_per_step": L_mean, "k": k_head, "multi_gpu": "replicas only",
+                   "l2": f"inputs larger than L2: tables {w.table_bytes() / 1e9:.2f} GB, {nd} distinct ID batches cycled"},
+        "by_k": {str(k): {"lookups_per_s": t / (m * 1e-3), "ms_per_step": m / args.steps} for k, (m, t) in by_k.items()},
+        "max_lag": lag,
+        "step_roofline": {"bound": "hbm", "achieved": step_gbs / world, "unit": "GB/s", "peak": peak,
+                          "frac": step_gbs / world / peak, "frac_of_nominal_8TBs": step_gbs / world / NOMINAL_HBM_GBS,
+                          "bytes_per_step": step_bytes, "peak_source": peak_src},
+        "roofline": {"bound": "hbm", "kernel": "bls_gather_pool_kernel", "achieved": ach, "peak": peak, "unit": "GB/s",
+                     "frac": ach / peak, "frac_of_nominal_8TBs": ach / NOMINAL_HBM_GBS,
+                     "traffic": traffic_record(os.path.join(ROOT, "paper_2512_19342_b200", "csrc", "bls_gather.cu"), w.name),
+                     "bytes_per_launch": gather_bytes, "ms_per_launch": ms_gather, "peak_source": peak_src},
+        "stage_ms_per_step": {"route": prof["ms_route"] / max(1, prof["calls"]), "gather_pool_return": ms_gather,
+                              "ring": prof["ms_ring"] / max(1, prof["calls"])},
+        "clocks": clocks, "e2e": e2e, "gpu_launches": launches,
+    }
+    if not args.no_cpu_baseline and world == 1:
+        result["cpu_baseline"] = cpu_baseline(w, inputs)
+    print(json.dumps(result))
+
+
+def main():
+    args = parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_mine(args)
+
+
+if __name__ == "__main__":
+    main()

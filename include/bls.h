@@ -156,6 +156,16 @@ bls_status_t bls_set_stall(bls_plan_t *plan, int rank, int64_t ns);
 /* Upper limit of any single device-side wait (default 2 s). */
 bls_status_t bls_set_wait_limit(bls_plan_t *plan, int64_t ns);
 
+/* Stage timing with CUDA events on the plan's stream.  While enabled, every
+ * bls_step/bls_drain records events around its three stages (up to 1024 calls
+ * are kept).  bls_profile_read synchronises the stream, adds up the recorded
+ * calls into milliseconds per stage (router kernels, the gather-pool-return
+ * kernel, gate + commit kernels), reports how many calls were summed and how
+ * many kernels they launched, and clears the record.  Any pointer may be NULL. */
+bls_status_t bls_profile(bls_plan_t *plan, int enable);
+bls_status_t bls_profile_read(bls_plan_t *plan, double *ms_route, double *ms_gather, double *ms_ring,
+                              int64_t *calls, int64_t *kernels);
+
 const char *bls_strerror(int status);
 
 /* ---- input generation helper (not part of the method) ----

@@ -23,7 +23,8 @@ _DTYPE = {torch.float32: BLS_F32, torch.bfloat16: BLS_BF16, torch.float16: BLS_F
 
 EXPORTS = ["bls_plan_bytes", "bls_plan", "bls_destroy", "bls_route", "bls_lookup", "bls_step",
            "bls_drain", "bls_step_host", "bls_drain_host", "bls_view", "bls_counters", "bls_status",
-           "bls_set_stall", "bls_set_wait_limit", "bls_strerror", "bls_fill_hash_table"]
+           "bls_set_stall", "bls_set_wait_limit", "bls_strerror", "bls_fill_hash_table",
+           "bls_profile", "bls_profile_read"]
 
 
 class BlsError(RuntimeError):
@@ -204,6 +205,20 @@ def bls_set_stall(plan: Plan, rank: int, ns: int) -> None:
 
 def bls_set_wait_limit(plan: Plan, ns: int) -> None:
     _check(lib().bls_set_wait_limit(plan.handle, C.c_int64(ns)), "bls_set_wait_limit")
+
+
+def bls_profile(plan: Plan, enable: bool) -> None:
+    _check(lib().bls_profile(plan.handle, int(enable)), "bls_profile")
+
+
+def bls_profile_read(plan: Plan) -> dict:
+    """Summed stage times (ms) of the calls recorded since the last read; synchronises."""
+    r, g, c = C.c_double(0), C.c_double(0), C.c_double(0)
+    n, kn = C.c_int64(0), C.c_int64(0)
+    _check(lib().bls_profile_read(plan.handle, C.byref(r), C.byref(g), C.byref(c), C.byref(n), C.byref(kn)),
+           "bls_profile_read")
+    return {"ms_route": r.value, "ms_gather": g.value, "ms_ring": c.value, "calls": n.value,
+            "kernels_total": kn.value}
 
 
 def bls_fill_hash_table(weight: torch.Tensor, seed: int, t: int,

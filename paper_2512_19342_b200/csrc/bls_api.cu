@@ -199,11 +199,74 @@ bls_status_t bls_plan(const bls_table_t *tables, int T, int part, int P, int loc
     return BLS_OK;
 }
 
-void bls_destroy(bls_plan_t *plan) { free(plan); }
+void bls_destroy(bls_plan_t *plan)
+{
+    if (!plan) return;
+    if (plan->prof_ev) {
+        for (int i = 0; i < BLS_PROF_MAX * 4; i++) cudaEventDestroy(plan->prof_ev[i]);
+        free(plan->prof_ev);
+    }
+    free(plan);
+}
+
+bls_status_t bls_profile(bls_plan_t *pl, int enable)
+{
+    if (!pl) return BLS_EINVAL;
+    pl->prof_on = enable ? 1 : 0;
+    return BLS_OK;
+}
+
+bls_status_t bls_profile_read(bls_plan_t *pl, double *ms_route, double *ms_gather, double *ms_ring,
+                              int64_t *calls, int64_t *kernels)
+{
+    if (!pl) return BLS_EINVAL;
+    if (cudaStreamSynchronize(pl->stream) != cudaSuccess) return BLS_ECUDA;
+    double r = 0, g = 0, c = 0;
+    for (int i = 0; i < pl->prof_n; i++) {
+        cudaEvent_t *ev = pl->prof_ev + (size_t)i * 4;
+        float a = 0, b = 0, d = 0;
+        if (cudaEventElapsedTime(&a, ev[0], ev[1]) != cudaSuccess ||
+            cudaEventElapsedTime(&b, ev[1], ev[2]) != cudaSuccess ||
+            cudaEventElapsedTime(&d, ev[2], ev[3]) != cudaSuccess)
+            return BLS_ECUDA;
+        r += a; g += b; c += d;
+    }
+    if (ms_route) *ms_route = r;
+    if (ms_gather) *ms_gather = g;
+    if (ms_ring) *ms_ring = c;
+    if (calls) *calls = pl->prof_n;
+    if (kernels) *kernels = pl->kernels_launched;
+    pl->prof_n = 0;
+    return BLS_OK;
+}
 
 static bls_status_t launch_check()
 {
     return cudaGetLastError() == cudaSuccess ? BLS_OK : BLS_ECUDA;
+}
+
+// One wave: gate -> router -> gather/pool/return -> commit, with optional stage events.
+static void enqueue_wave(bls_plan_t *pl, int mode, long long t_last, long long floor_, int k,
+                         const int *ids, const int *off, long long n_ids)
+{
+    cudaEvent_t *ev = nullptr;
+    if (pl->prof_on && pl->prof_n < BLS_PROF_MAX) {
+        if (!pl->prof_ev) {
+            pl->prof_ev = (cudaEvent_t *)calloc((size_t)BLS_PROF_MAX * 4, sizeof(cudaEvent_t));
+            if (pl->prof_ev)
+                for (int i = 0; i < BLS_PROF_MAX * 4; i++) cudaEventCreate(&pl->prof_ev[i]);
+        }
+        if (pl->prof_ev) ev = pl->prof_ev + (size_t)pl->prof_n++ * 4;
+    }
+    if (ev) cudaEventRecord(ev[0], pl->stream);
+    bls_launch_gate(pl, mode, t_last, floor_, k, ids, off, n_ids);
+    bls_launch_route(pl);
+    if (ev) cudaEventRecord(ev[1], pl->stream);
+    bls_launch_gather(pl);
+    if (ev) cudaEventRecord(ev[2], pl->stream);
+    bls_launch_commit(pl);
+    if (ev) cudaEventRecord(ev[3], pl->stream);
+    pl->kernels_launched += 3 + bls_route_kernels(pl);
 }
 
 static const float *slot_out(const bls_plan_t *pl, long long iter)
@@ -219,6 +282,7 @@ bls_status_t bls_route(bls_plan_t *pl, int64_t iter, const int32_t *ids, const i
     bls_launch_gate(pl, BLS_MODE_ROUTE_ONLY, iter, -1, 0, ids, offsets, n_ids);
     bls_launch_route(pl);
     bls_launch_commit(pl);
+    pl->kernels_launched += 2 + bls_route_kernels(pl);
     pl->routed_only = iter;
     pl->t_next = iter + 1;
     return launch_check();
@@ -231,6 +295,7 @@ bls_status_t bls_lookup(bls_plan_t *pl, int64_t iter)
     bls_launch_gate(pl, BLS_MODE_LOOKUP_ONLY, iter, -1, 0, nullptr, nullptr, 0);
     bls_launch_gather(pl);
     bls_launch_commit(pl);
+    pl->kernels_launched += 3;
     pl->routed_only = -1;
     pl->t_handed = iter + 1;
     return launch_check();
@@ -244,10 +309,7 @@ bls_status_t bls_step(bls_plan_t *pl, int k, const int32_t *ids, const int32_t *
     if (pl->k_cur >= 0 && pl->k_cur != k && pl->t_handed != pl->t_next) return BLS_ESTATE;
     pl->k_cur = k;
     const long long t = pl->t_next++;
-    bls_launch_gate(pl, BLS_MODE_STEP, t, t - k, k, ids, offsets, n_ids);
-    bls_launch_route(pl);
-    bls_launch_gather(pl);
-    bls_launch_commit(pl);
+    enqueue_wave(pl, BLS_MODE_STEP, t, t - k, k, ids, offsets, n_ids);
     if (t - k >= 0) {
         *out = slot_out(pl, t - k);
         *out_iter = t - k;
@@ -270,10 +332,10 @@ bls_status_t bls_drain(bls_plan_t *pl, const float **out, int64_t *out_iter)
         return BLS_OK;
     }
     const long long f = pl->t_handed;
-    bls_launch_gate(pl, BLS_MODE_DRAIN, pl->t_next - 1, f, pl->k_cur < 0 ? 0 : pl->k_cur, nullptr, nullptr, 0);
-    bls_launch_route(pl);
-    bls_launch_gather(pl);
-    bls_launch_commit(pl);
+    // Without injected delays every rank completes an iteration in the step that
+    // issues it, so the outstanding iterations are already complete on the stream.
+    if (pl->any_stall)
+        enqueue_wave(pl, BLS_MODE_DRAIN, pl->t_next - 1, f, pl->k_cur < 0 ? 0 : pl->k_cur, nullptr, nullptr, 0);
     *out = slot_out(pl, f);
     *out_iter = f;
     pl->t_handed = f + 1;
@@ -373,6 +435,7 @@ bls_status_t bls_set_stall(bls_plan_t *pl, int rank, int64_t ns)
 {
     if (!pl || rank < 0 || rank >= pl->prm.P || ns < 0) return BLS_EINVAL;
     unsigned long long v = (unsigned long long)ns;
+    if (ns > 0) pl->any_stall = 1;
     return cudaMemcpyAsync(&pl->prm.dev->stall_ns[rank], &v, sizeof(v), cudaMemcpyHostToDevice,
                            pl->stream) == cudaSuccess &&
                    cudaStreamSynchronize(pl->stream) == cudaSuccess

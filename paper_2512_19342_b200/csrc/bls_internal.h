@@ -88,7 +88,14 @@ struct bls_plan {
     long long routed_only;  // iteration routed by bls_route and not yet looked up, or -1
     size_t bytes;
     int sm_count;
+    // optional stage timing (events are created on first use, 4 per recorded call)
+    int prof_on;
+    int prof_n;
+    cudaEvent_t *prof_ev;
+    long long kernels_launched;   // total kernels enqueued through this plan
+    int any_stall;                // a delay was injected at some point: ranks may be out of lockstep
 };
+#define BLS_PROF_MAX 1024
 
 // kernel launchers (defined in the .cu files)
 void bls_launch_gate(const bls_plan_t *pl, int mode, long long t_last, long long forced_floor, int k,
@@ -96,4 +103,4 @@ void bls_launch_gate(const bls_plan_t *pl, int mode, long long t_last, long long
 void bls_launch_commit(const bls_plan_t *pl);
 void bls_launch_route(const bls_plan_t *pl);
 void bls_launch_gather(const bls_plan_t *pl);
-void bls_launch_init(const bls_plan_t *pl, const BlsDev *host_dev);
+int bls_route_kernels(const bls_plan_t *pl);   // kernels bls_launch_route enqueues

@@ -280,6 +280,8 @@ __global__ void __launch_bounds__(BLS_ROUTE_TB) bls_rw_scatter_kernel(BlsParams 
     }
 }
 
+int bls_route_kernels(const bls_plan_t *pl) { return pl->prm.part == BLS_PART_TABLE_RR ? 2 : 3; }
+
 void bls_launch_route(const bls_plan_t *pl)
 {
     const BlsParams &p = pl->prm;
