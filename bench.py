@@ -44,6 +44,7 @@ def parse_args():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--tables", type=int, default=0, help="keep only the first N tables (reduced profiling case)")
+    ap.add_argument("--tune", default="", help="bags_per_run,rows_in_flight for the gather kernel (0 = default)")
     ap.add_argument("--ks", default="", help="comma-separated bounds to time instead of the workload's own")
     return ap.parse_args()
 
@@ -308,6 +309,9 @@ def run_mine(args):
     Ls = [len(i) for i, _ in inputs]
     k_max = max(w.ks)
     plan = bls.bls_plan(tabs, w.partition, w.P, w.local_batch, k_max, capacity(w, inputs))
+
+    if args.tune:
+        bls.bls_set_tuning(plan, *[int(x) for x in args.tune.split(",")])
 
     def loop(k, steps):
         for t in range(steps):

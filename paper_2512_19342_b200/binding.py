@@ -24,7 +24,7 @@ _DTYPE = {torch.float32: BLS_F32, torch.bfloat16: BLS_BF16, torch.float16: BLS_F
 EXPORTS = ["bls_plan_bytes", "bls_plan", "bls_destroy", "bls_route", "bls_lookup", "bls_step",
            "bls_drain", "bls_step_host", "bls_drain_host", "bls_view", "bls_counters", "bls_status",
            "bls_set_stall", "bls_set_wait_limit", "bls_strerror", "bls_fill_hash_table",
-           "bls_profile", "bls_profile_read"]
+           "bls_profile", "bls_profile_read", "bls_set_tuning"]
 
 
 class BlsError(RuntimeError):
@@ -205,6 +205,10 @@ def bls_set_stall(plan: Plan, rank: int, ns: int) -> None:
 
 def bls_set_wait_limit(plan: Plan, ns: int) -> None:
     _check(lib().bls_set_wait_limit(plan.handle, C.c_int64(ns)), "bls_set_wait_limit")
+
+
+def bls_set_tuning(plan: Plan, bags_per_run: int = 0, rows_in_flight: int = 0) -> None:
+    _check(lib().bls_set_tuning(plan.handle, bags_per_run, rows_in_flight), "bls_set_tuning")
 
 
 def bls_profile(plan: Plan, enable: bool) -> None:

@@ -21,7 +21,7 @@ bls_status_t check_shape(const bls_table_t *tables, int T, int part, int P, int 
                          int64_t cap)
 {
     if (!tables || T < 1 || P < 1 || P > BLS_MAX_RANKS || b < 1 || k_max < 0 ||
-        k_max + 1 > BLS_MAX_SLOTS || cap < 1 || cap > 0x7fffffff)
+        k_max + 1 > BLS_MAX_SLOTS || cap < 1 || cap > 0x7ffffff0)
         return BLS_EINVAL;
     if (part != BLS_PART_TABLE_RR && part != BLS_PART_ROW_BLOCK) return BLS_EINVAL;
     const int D = tables[0].dim, dt = tables[0].dtype;
@@ -47,7 +47,7 @@ void fill_params(BlsParams &p, const bls_table_t *tables, int T, int part, int P
     p.lanes = p.row_bytes / 16;
     p.NI = part == BLS_PART_TABLE_RR ? T : T * P;
     p.NQ = p.NI * b;
-    p.cap = (int)cap;
+    p.cap = (int)((cap + 3) / 4 * 4);          // every rank's send buffer starts on a 16-byte boundary
     p.tiles_per_table = (b + BLS_ROUTE_TB - 1) / BLS_ROUTE_TB;
     p.NT = T * p.tiles_per_table;
     p.sub_stride = (long long)align_up((size_t)p.NQ + 1, 4);
@@ -141,6 +141,12 @@ bls_status_t bls_plan(const bls_table_t *tables, int T, int part, int P, int loc
     pl->k_cur = -1;
     pl->routed_only = -1;
     pl->bytes = L.total;
+    {   // runs of about 320 rows: long enough to amortise the start of a run, short enough to balance
+        double avg = (double)max_ids_per_rank / ((double)p.NI * local_batch);
+        int R = (int)(320.0 / (avg < 0.5 ? 0.5 : avg) + 0.5);
+        pl->bags_per_run = R < 4 ? 4 : (R > 64 ? 64 : R);
+        pl->rows_in_flight = 4;
+    }
     int devid = 0;
     if (!cuda_ok(cudaGetDevice(&devid)) ||
         !cuda_ok(cudaDeviceGetAttribute(&pl->sm_count, cudaDevAttrMultiProcessorCount, devid))) {
@@ -441,6 +447,15 @@ bls_status_t bls_set_stall(bls_plan_t *pl, int rank, int64_t ns)
                    cudaStreamSynchronize(pl->stream) == cudaSuccess
                ? BLS_OK
                : BLS_ECUDA;
+}
+
+bls_status_t bls_set_tuning(bls_plan_t *pl, int bags_per_run, int rows_in_flight)
+{
+    if (!pl || bags_per_run < 0 || bags_per_run > 4096 || (rows_in_flight != 0 && rows_in_flight != 4 && rows_in_flight != 8))
+        return BLS_EINVAL;
+    if (bags_per_run) pl->bags_per_run = bags_per_run;
+    if (rows_in_flight) pl->rows_in_flight = rows_in_flight;
+    return BLS_OK;
 }
 
 bls_status_t bls_set_wait_limit(bls_plan_t *pl, int64_t ns)

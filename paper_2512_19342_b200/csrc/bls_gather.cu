@@ -3,148 +3,244 @@
 // straight into the requester's output slot out[src][s][t][:], so the pooled
 // vectors never make a round trip through memory.
 //
-// HBM-bound random row reads: a group of LANES = row_bytes/16 lanes owns one
-// sub-bag; every lane keeps one 16-byte piece of the row, loads of up to 8 rows
-// are issued back to back before the first add (memory-level parallelism), IDs
-// are read coalesced and broadcast with shuffles.  Sub-bags are visited
-// table-major, so the SMs work on one table at a time and the Zipf-hot rows of
-// that table stay in L1/L2.  IDs and outputs use streaming loads/stores so they
-// do not evict table rows.
+// The work is random row reads, bound by memory latency unless enough loads are in
+// flight.  A group of LANES = row_bytes/16 lanes streams a *run* of consecutive
+// sub-bags of one (owner, table, requester) chunk: their IDs are contiguous in the
+// requester's packed send buffer, so the group walks one ID stream and keeps
+// batches of U row loads in flight across bag boundaries (two batches are
+// outstanding while a third batch's IDs are being fetched, 16 bytes at a time from
+// aligned addresses); a bag boundary only costs a store of the accumulator.  Rows of one bag are added in their original
+// order, so the result does not depend on how runs are cut.  Runs are handed out
+// through an atomic counter in table-major order: at any moment the SMs work on
+// one or two tables, whose Zipf-hot rows stay in L1/L2.  IDs and outputs use
+// streaming loads/stores so that they do not evict table rows.
 #include <cuda_bf16.h>
 #include <cuda_fp16.h>
 #include "bls_internal.h"
 
+// fp32 accumulators as packed pairs: sm_100 adds two fp32 lanes per instruction
+// (round-to-nearest, identical to two scalar adds).
 template <int DT> struct Acc;
 template <> struct Acc<BLS_F32> {
-    float v[4];
-    __device__ __forceinline__ void zero() { v[0] = v[1] = v[2] = v[3] = 0.f; }
+    static constexpr int N = 4;
+    float2 a, b;
+    __device__ __forceinline__ void zero() { a = b = make_float2(0.f, 0.f); }
     __device__ __forceinline__ void add(const uint4 &u)
     {
-        v[0] += __uint_as_float(u.x); v[1] += __uint_as_float(u.y);
-        v[2] += __uint_as_float(u.z); v[3] += __uint_as_float(u.w);
+        a = __fadd2_rn(a, make_float2(__uint_as_float(u.x), __uint_as_float(u.y)));
+        b = __fadd2_rn(b, make_float2(__uint_as_float(u.z), __uint_as_float(u.w)));
     }
-    static constexpr int N = 4;
+    __device__ __forceinline__ float4 lo() const { return make_float4(a.x, a.y, b.x, b.y); }
+    __device__ __forceinline__ float4 hi() const { return make_float4(0.f, 0.f, 0.f, 0.f); }
 };
 template <> struct Acc<BLS_BF16> {
-    float v[8];
-    __device__ __forceinline__ void zero() { for (int i = 0; i < 8; i++) v[i] = 0.f; }
-    __device__ __forceinline__ void add(const uint4 &u)
-    {   // a bf16 is the upper half of an fp32: widening is exact
-        v[0] += __uint_as_float(u.x << 16); v[1] += __uint_as_float(u.x & 0xffff0000u);
-        v[2] += __uint_as_float(u.y << 16); v[3] += __uint_as_float(u.y & 0xffff0000u);
-        v[4] += __uint_as_float(u.z << 16); v[5] += __uint_as_float(u.z & 0xffff0000u);
-        v[6] += __uint_as_float(u.w << 16); v[7] += __uint_as_float(u.w & 0xffff0000u);
-    }
     static constexpr int N = 8;
-};
-template <> struct Acc<BLS_F16> {
-    float v[8];
-    __device__ __forceinline__ void zero() { for (int i = 0; i < 8; i++) v[i] = 0.f; }
+    float2 a, b, c, d;
+    __device__ __forceinline__ void zero() { a = b = c = d = make_float2(0.f, 0.f); }
+    // a bf16 is the upper half of an fp32: widening is exact
+    static __device__ __forceinline__ float2 w(unsigned u)
+    {
+        return make_float2(__uint_as_float(u << 16), __uint_as_float(u & 0xffff0000u));
+    }
     __device__ __forceinline__ void add(const uint4 &u)
     {
-        const unsigned w[4] = {u.x, u.y, u.z, u.w};
-        #pragma unroll
-        for (int i = 0; i < 4; i++) {
-            float2 f = __half22float2(*reinterpret_cast<const __half2 *>(&w[i]));
-            v[2 * i] += f.x; v[2 * i + 1] += f.y;
-        }
+        a = __fadd2_rn(a, w(u.x)); b = __fadd2_rn(b, w(u.y));
+        c = __fadd2_rn(c, w(u.z)); d = __fadd2_rn(d, w(u.w));
     }
+    __device__ __forceinline__ float4 lo() const { return make_float4(a.x, a.y, b.x, b.y); }
+    __device__ __forceinline__ float4 hi() const { return make_float4(c.x, c.y, d.x, d.y); }
+};
+template <> struct Acc<BLS_F16> {
     static constexpr int N = 8;
+    float2 a, b, c, d;
+    __device__ __forceinline__ void zero() { a = b = c = d = make_float2(0.f, 0.f); }
+    static __device__ __forceinline__ float2 w(unsigned u)
+    {
+        return __half22float2(*reinterpret_cast<const __half2 *>(&u));
+    }
+    __device__ __forceinline__ void add(const uint4 &u)
+    {
+        a = __fadd2_rn(a, w(u.x)); b = __fadd2_rn(b, w(u.y));
+        c = __fadd2_rn(c, w(u.z)); d = __fadd2_rn(d, w(u.w));
+    }
+    __device__ __forceinline__ float4 lo() const { return make_float4(a.x, a.y, b.x, b.y); }
+    __device__ __forceinline__ float4 hi() const { return make_float4(c.x, c.y, d.x, d.y); }
 };
 
-__device__ __forceinline__ void red_add_v4(float *addr, float a, float b, float c, float d)
+__device__ __forceinline__ void red_add_v4(float *addr, float4 v)
 {
-    asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(addr), "f"(a), "f"(b), "f"(c), "f"(d)
+    asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(addr), "f"(v.x), "f"(v.y), "f"(v.z),
+                 "f"(v.w)
                  : "memory");
 }
 
-template <int LANES, int DT, bool ROWWISE>
-__global__ void __launch_bounds__(256) bls_gather_pool_kernel(BlsParams p, long long n_work)
+template <int DT, bool ROWWISE>
+__device__ __forceinline__ void flush(float *o, const Acc<DT> &acc, bool nonempty)
 {
-    constexpr int U = LANES < 8 ? LANES : 8;           // rows in flight per group and batch
-    constexpr int GROUPS = 256 / LANES;
-    const int lane = threadIdx.x % LANES;
-    const int gidx = threadIdx.x / LANES;
-    const unsigned gmask = LANES == 32 ? 0xffffffffu
-                                       : (((1u << LANES) - 1u) << ((threadIdx.x & 31) / LANES * LANES));
-    const long long Pb = (long long)p.P * p.b;
-    const BlsDev *dev = p.dev;
-
-    for (long long w = (long long)blockIdx.x * GROUPS + gidx; w < n_work; w += (long long)gridDim.x * GROUPS) {
-        const int i = (int)(w / Pb);                   // (owner, table) pair, owner-major
-        const int rem = (int)(w - (long long)i * Pb);
-        const int src = rem / p.b, s = rem - src * p.b;
-        const BlsPairDesc pr = p.pair[i];
-        const long long j = dev->serve_iter[pr.dst];
-        if (j < 0) continue;                           // this owner does not serve in this wave
-        const int slot = (int)(j % p.S);
-        const int *ss = p.sub_start + ((size_t)slot * p.P + src) * (size_t)p.sub_stride + (size_t)i * p.b + s;
-        int st = ss[0], en = ss[1];
-        st = min(max(st, 0), p.cap);
-        en = min(max(en, st), p.cap);
-        if (ROWWISE && en == st) continue;             // nothing to add
-        const int *sb = p.sendbuf + ((size_t)slot * p.P + src) * (size_t)p.cap;
-        const uint4 *base = reinterpret_cast<const uint4 *>(pr.base);
-        const unsigned nrows_m1 = (unsigned)pr.nrows - 1u;
-
-        Acc<DT> acc;
-        acc.zero();
-        for (int c0 = st; c0 < en; c0 += LANES) {
-            const int n = min(LANES, en - c0);
-            int my = (lane < n) ? __ldcs(sb + c0 + lane) : 0;
-            #pragma unroll 1
-            for (int u0 = 0; u0 < n; u0 += U) {
-                uint4 v[U];
-                #pragma unroll
-                for (int u = 0; u < U; u++) {
-                    unsigned row = (unsigned)__shfl_sync(gmask, my, u0 + u, LANES);
-                    row = min(row, nrows_m1);
-                    if (u0 + u < n) v[u] = __ldg(base + (size_t)row * LANES + lane);
-                    else v[u] = make_uint4(0u, 0u, 0u, 0u);
-                }
-                #pragma unroll
-                for (int u = 0; u < U; u++) acc.add(v[u]);
-            }
-        }
-        float *o = p.out + (size_t)slot * p.out_slot_elems +
-                   (((size_t)src * p.b + s) * p.T + pr.t) * p.D + lane * Acc<DT>::N;
-        if (ROWWISE) {
-            red_add_v4(o, acc.v[0], acc.v[1], acc.v[2], acc.v[3]);
-            if (Acc<DT>::N == 8) red_add_v4(o + 4, acc.v[4], acc.v[5], acc.v[6], acc.v[7]);
-        } else {
-            __stcs(reinterpret_cast<float4 *>(o), make_float4(acc.v[0], acc.v[1], acc.v[2], acc.v[3]));
-            if (Acc<DT>::N == 8)
-                __stcs(reinterpret_cast<float4 *>(o) + 1, make_float4(acc.v[4], acc.v[5], acc.v[6], acc.v[7]));
-        }
+    if (ROWWISE) {
+        if (!nonempty) return;                         // nothing to add to the requester's sum
+        red_add_v4(o, acc.lo());
+        if (Acc<DT>::N == 8) red_add_v4(o + 4, acc.hi());
+    } else {
+        __stcs(reinterpret_cast<float4 *>(o), acc.lo());
+        if (Acc<DT>::N == 8) __stcs(reinterpret_cast<float4 *>(o) + 1, acc.hi());
     }
 }
 
-template <int LANES, int DT>
+template <int LANES, int DT, bool ROWWISE, int U>
+__global__ void __launch_bounds__(256, (U >= 8 ? 2 : 3))
+bls_gather_pool_kernel(BlsParams p, int R, int runs_per_chunk, int n_runs)
+{
+    constexpr int GPW = 32 / LANES;                    // groups (runs) per warp
+    constexpr int Q = U / 4;                           // 16-byte ID quads per batch
+    const int lane = threadIdx.x % LANES;
+    const int g = (threadIdx.x & 31) / LANES;
+    BlsDev *dev = p.dev;
+    const size_t bag_stride = (size_t)p.T * p.D;       // floats between consecutive samples in out
+
+    int base = 0;
+    if ((threadIdx.x & 31) == 0) base = atomicAdd(&dev->work_ctr, GPW);
+    base = __shfl_sync(0xffffffffu, base, 0);
+    while (base < n_runs) {
+        int next_base = 0;                             // grab the next runs now, use them later
+        if ((threadIdx.x & 31) == 0) next_base = atomicAdd(&dev->work_ctr, GPW);
+        const int run = base + g;
+        if (run < n_runs) {
+            const int chunk = run / runs_per_chunk;    // (pair, requester), pair-major
+            const int s0 = (run - chunk * runs_per_chunk) * R;
+            const int i = chunk / p.P, src = chunk - i * p.P;
+            const BlsPairDesc pr = p.pair[i];
+            const long long j = dev->serve_iter[pr.dst];
+            if (j >= 0) {                              // else: this owner does not serve in this wave
+                const int slot = (int)(j % p.S);
+                const int nb = min(R, p.b - s0);
+                const int *ss = p.sub_start + ((size_t)slot * p.P + src) * (size_t)p.sub_stride + (size_t)i * p.b + s0;
+                const int p0 = min(max(ss[0], 0), p.cap);
+                const int n = min(max(ss[nb], p0), p.cap) - p0;          // rows in this run
+                // The ID stream is read in aligned 16-byte quads and processed in whole batches
+                // of U rows: stream coordinate y = a + x, where x counts the run's rows and
+                // a = p0 mod 4.  The a IDs before the run and the IDs after it up to the end of
+                // the last batch belong to other bags (or to nobody); their rows are loaded
+                // (clamped, so always in bounds) and accumulated into a "bag" that is never
+                // stored.  That keeps the inner loop free of validity predicates.
+                const int a = p0 & 3;
+                const int yend = a + n;
+                const int org = a - p0;                // y coordinate of send-buffer position 0
+                // bag c of the run ends at bag_end(c); c = -1 is the part before the run, c = nb the part after
+                auto bag_end = [&](int c) {
+                    return c < 0 ? a : c < nb - 1 ? min(max(ss[c + 1] + org, a), yend) : c == nb - 1 ? yend : 0x7fffffff;
+                };
+                int cur = -1;
+                int e_cur = a, e_nxt = bag_end(0);
+                int start = 0;                         // y where the current bag started
+                const int4 *sq = reinterpret_cast<const int4 *>(
+                    p.sendbuf + ((size_t)slot * p.P + src) * (size_t)p.cap + (p0 - a));
+                const uint4 *rowbase = reinterpret_cast<const uint4 *>(pr.base) + lane;
+                const unsigned nrows_m1 = (unsigned)pr.nrows - 1u;
+                float *o = p.out + (size_t)slot * p.out_slot_elems +
+                           (((size_t)src * p.b + s0) * p.T + pr.t) * p.D + lane * Acc<DT>::N;
+
+                Acc<DT> acc;
+                acc.zero();
+                int4 ida[Q], idb[Q];                   // IDs of the next batch for va / for vb
+                uint4 va[U], vb[U];
+                const int nbat = (yend + U - 1) / U;
+
+                auto load_ids = [&](int4(&idq)[Q], int k) {
+                    if (k >= nbat) return;
+                    #pragma unroll
+                    for (int q = 0; q < Q; q++) idq[q] = __ldcs(sq + k * Q + q);
+                };
+                auto issue = [&](uint4(&v)[U], const int4(&idq)[Q], int k) {
+                    if (k >= nbat) return;
+                    #pragma unroll
+                    for (int u = 0; u < U; u++) {
+                        const unsigned id = (unsigned)(&idq[u / 4].x)[u & 3];
+                        v[u] = __ldg(rowbase + (size_t)min(id, nrows_m1) * LANES);
+                    }
+                };
+                auto consume = [&](const uint4(&v)[U], int k) {
+                    if (k >= nbat) return;
+                    #pragma unroll
+                    for (int u = 0; u < U; u++) {
+                        const int y = k * U + u;
+                        while (y == e_cur) {           // bags that end here (possibly empty ones)
+                            if (cur >= 0) {
+                                flush<DT, ROWWISE>(o, acc, y > start);
+                                o += bag_stride;
+                            }
+                            acc.zero();
+                            cur++;
+                            start = y;
+                            e_cur = e_nxt;
+                            e_nxt = bag_end(cur + 1);
+                        }
+                        acc.add(v[u]);
+                    }
+                };
+
+                // Pipeline: the IDs of a batch are fetched two batches before its rows are
+                // requested, and its rows one batch before they are added, so that neither the ID
+                // latency nor the row latency sits on the critical path.
+                load_ids(ida, 0);
+                load_ids(idb, 1);
+                issue(va, ida, 0);
+                load_ids(ida, 2);
+                for (int k = 0; k < nbat; k += 2) {
+                    issue(vb, idb, k + 1);
+                    load_ids(idb, k + 3);
+                    consume(va, k);
+                    issue(va, ida, k + 2);
+                    load_ids(ida, k + 4);
+                    consume(vb, k + 1);
+                }
+                // bags not closed by a row after them: the last one when the run ends on a batch
+                // boundary, and everything when the run has no rows at all
+                if (cur < 0) { cur = 0; start = yend; acc.zero(); }
+                for (; cur < nb; cur++) {
+                    flush<DT, ROWWISE>(o, acc, yend > start);
+                    o += bag_stride;
+                    acc.zero();
+                    start = yend;
+                }
+            }
+        }
+        __syncwarp();
+        base = __shfl_sync(0xffffffffu, next_base, 0);
+    }
+}
+
+template <int LANES, int DT, int U>
 static void launch_gather(const bls_plan_t *pl)
 {
     const BlsParams &p = pl->prm;
-    const long long n_work = (long long)p.NI * p.P * p.b;
-    const int groups = 256 / LANES;
-    long long blocks = (n_work + groups - 1) / groups;
-    const long long cap_blocks = (long long)pl->sm_count * 64;
-    if (blocks > cap_blocks) blocks = cap_blocks;
-    if (blocks < 1) blocks = 1;
+    const int R = pl->bags_per_run;
+    const int rpc = (p.b + R - 1) / R;
+    const long long n_runs = (long long)p.NI * p.P * rpc;
+    const int blocks = pl->sm_count * 8;               // more than fit: late blocks find the counter exhausted
     if (p.part == BLS_PART_ROW_BLOCK)
-        bls_gather_pool_kernel<LANES, DT, true><<<(unsigned)blocks, 256, 0, pl->stream>>>(p, n_work);
+        bls_gather_pool_kernel<LANES, DT, true, U><<<blocks, 256, 0, pl->stream>>>(p, R, rpc, (int)n_runs);
     else
-        bls_gather_pool_kernel<LANES, DT, false><<<(unsigned)blocks, 256, 0, pl->stream>>>(p, n_work);
+        bls_gather_pool_kernel<LANES, DT, false, U><<<blocks, 256, 0, pl->stream>>>(p, R, rpc, (int)n_runs);
+}
+
+template <int LANES, int DT>
+static void launch_gather_u(const bls_plan_t *pl)
+{
+    if (pl->rows_in_flight >= 8) launch_gather<LANES, DT, 8>(pl);
+    else launch_gather<LANES, DT, 4>(pl);
 }
 
 template <int DT>
 static void launch_gather_dt(const bls_plan_t *pl)
 {
     switch (pl->prm.lanes) {
-    case 1: launch_gather<1, DT>(pl); break;
-    case 2: launch_gather<2, DT>(pl); break;
-    case 4: launch_gather<4, DT>(pl); break;
-    case 8: launch_gather<8, DT>(pl); break;
-    case 16: launch_gather<16, DT>(pl); break;
-    default: launch_gather<32, DT>(pl); break;
+    case 1: launch_gather_u<1, DT>(pl); break;
+    case 2: launch_gather_u<2, DT>(pl); break;
+    case 4: launch_gather_u<4, DT>(pl); break;
+    case 8: launch_gather_u<8, DT>(pl); break;
+    case 16: launch_gather_u<16, DT>(pl); break;
+    default: launch_gather_u<32, DT>(pl); break;
     }
 }
 

@@ -34,7 +34,7 @@ struct BlsDev {
     unsigned long long wait_limit_ns;
     long long max_lag;                            // max over time of newest posted - oldest incomplete
     int status;                                   // OR of BLS_ST_* bits
-    int pad;
+    int work_ctr;                                 // next run of the gather kernel (reset by the gate)
 };
 
 struct BlsTableDesc {
@@ -94,6 +94,8 @@ struct bls_plan {
     cudaEvent_t *prof_ev;
     long long kernels_launched;   // total kernels enqueued through this plan
     int any_stall;                // a delay was injected at some point: ranks may be out of lockstep
+    int bags_per_run;             // gather kernel: consecutive sub-bags streamed by one lane group
+    int rows_in_flight;           // gather kernel: row loads per batch (4 or 8)
 };
 #define BLS_PROF_MAX 1024
 
