@@ -217,7 +217,9 @@ static void launch_gather(const bls_plan_t *pl)
     const int R = pl->bags_per_run;
     const int rpc = (p.b + R - 1) / R;
     const long long n_runs = (long long)p.NI * p.P * rpc;
-    const int blocks = pl->sm_count * 8;               // more than fit: late blocks find the counter exhausted
+    // more blocks than fit at once (late ones find the counter exhausted), fewer for small workloads
+    const long long want = (n_runs + 8 * (32 / LANES) - 1) / (8 * (32 / LANES));
+    const int blocks = (int)(want < 1 ? 1 : (want > pl->sm_count * 8 ? pl->sm_count * 8 : want));
     if (p.part == BLS_PART_ROW_BLOCK)
         bls_gather_pool_kernel<LANES, DT, true, U><<<blocks, 256, 0, pl->stream>>>(p, R, rpc, (int)n_runs);
     else
