@@ -181,6 +181,38 @@ const char *bls_strerror(int status);
 bls_status_t bls_fill_hash_table(void *weight, int64_t rows, int32_t dim, int32_t dtype,
                                  uint64_t seed, int32_t t, void *cuda_stream);
 
+/* ---- allocation-free router (the paper has no counterpart: this entry point
+ * exists for deployment reasons only) ----
+ * Step (1) for table-wise round-robin placement, for callers that cannot
+ * allocate device memory and therefore cannot provide a plan's workspace: code
+ * embedded in a server or framework that owns all device memory, plugins that
+ * receive fixed buffers, and loops where cudaMalloc's device-wide
+ * synchronisation or its failure under a full pool is unacceptable.  The call
+ * uses no workspace and calls no allocator: its only scratch (the start of each
+ * (requester, table) chunk) lives in a 128 KiB static device array inside the
+ * library, which every GPU that loads the library holds until the process exits.
+ *
+ *   table_rows  device, int64 [T]: table heights (for the ID range check)
+ *   ids/offsets device, as everywhere else; n_ids = offsets[P*T*local_batch]
+ *   sendcounts, sdispls  device out, int32 [P][P] indexed [src][dst]
+ *   sendbuf     device out, int32 [P][cap]: rank src's packed send buffer at src*cap
+ *   sub_start   device out, int32 [P][T*local_batch + 1], ordered (dst, table, sample)
+ *   status      device out, one int32: 0, or an OR of 1 (malformed offsets),
+ *               2 (cap too small), 4 (ID out of range, replaced by row 0)
+ * Results are identical to bls_route + bls_view on a table-wise plan.
+ *
+ * Limits and rules: P * (T + 1) <= 32768, else BLS_ENOSPC.  The first call on a
+ * device looks up the scratch array's device address (with that device current);
+ * make that first call before any stream capture.  All calls on a device share
+ * the array, which keeps the last call's contents; the part in use is cleared at
+ * the start of each call.  Calls whose GPU work may overlap (other streams or
+ * host threads) race on it: serialise them.  Asynchronous on `cuda_stream`. */
+bls_status_t bls_route_table_rr_static(const int64_t *table_rows, int T, int P, int local_batch,
+                                       const int32_t *ids, const int32_t *offsets, int64_t n_ids,
+                                       int32_t *sendcounts, int32_t *sdispls, int32_t *sendbuf,
+                                       int64_t cap, int32_t *sub_start, int32_t *status,
+                                       void *cuda_stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -24,7 +24,7 @@ _DTYPE = {torch.float32: BLS_F32, torch.bfloat16: BLS_BF16, torch.float16: BLS_F
 EXPORTS = ["bls_plan_bytes", "bls_plan", "bls_destroy", "bls_route", "bls_lookup", "bls_step",
            "bls_drain", "bls_step_host", "bls_drain_host", "bls_view", "bls_counters", "bls_status",
            "bls_set_stall", "bls_set_wait_limit", "bls_strerror", "bls_fill_hash_table",
-           "bls_profile", "bls_profile_read", "bls_set_tuning"]
+           "bls_profile", "bls_profile_read", "bls_set_tuning", "bls_route_table_rr_static"]
 
 
 class BlsError(RuntimeError):
@@ -231,3 +231,21 @@ def bls_fill_hash_table(weight: torch.Tensor, seed: int, t: int,
                                      C.c_int32(weight.shape[1]), _DTYPE[weight.dtype],
                                      C.c_uint64(seed & ((1 << 64) - 1)), C.c_int32(t), _stream_ptr(stream)),
            "bls_fill_hash_table")
+
+
+def bls_route_table_rr_static(table_rows: torch.Tensor, P: int, local_batch: int, ids: torch.Tensor,
+                              offsets: torch.Tensor, sendcounts: torch.Tensor, sdispls: torch.Tensor,
+                              sendbuf: torch.Tensor, sub_start: torch.Tensor, status: torch.Tensor,
+                              stream: Optional[torch.cuda.Stream] = None) -> None:
+    """Table-wise router without a plan or workspace, for callers that cannot allocate
+    device memory (the scratch is a static array inside the library).  Every tensor is
+    the caller's: table_rows int64 [T]; sendcounts/sdispls int32 [P][P]; sendbuf int32
+    [P][cap]; sub_start int32 [P][T*local_batch+1]; status int32 [1].  This wrapper
+    allocates nothing either."""
+    T = table_rows.numel()
+    _check(lib().bls_route_table_rr_static(
+        C.c_void_p(table_rows.data_ptr()), T, P, local_batch, C.c_void_p(ids.data_ptr()),
+        C.c_void_p(offsets.data_ptr()), C.c_int64(ids.numel()), C.c_void_p(sendcounts.data_ptr()),
+        C.c_void_p(sdispls.data_ptr()), C.c_void_p(sendbuf.data_ptr()), C.c_int64(sendbuf.shape[1]),
+        C.c_void_p(sub_start.data_ptr()), C.c_void_p(status.data_ptr()), _stream_ptr(stream)),
+        "bls_route_table_rr_static")
