@@ -73,10 +73,13 @@ typedef struct {
  *   recvcounts/rdispls  [P][P] indexed [dst][src]   (valid once the iteration has been looked up)
  *   sendbuf             rank src's packed send buffer starts at sendbuf + src*sendbuf_stride;
  *                       owner-local rows, sorted by dst, ties in original order
- *   sub_start           rank src's array starts at sub_start + src*sub_stride and has
- *                       subbags_per_rank + 1 entries: start position (in src's send buffer) of
- *                       each sub-bag, ordered (dst, table, sample); consecutive differences are the
- *                       sub-bag lengths the owner uses to rebuild bag boundaries
+ *   sub_start           rank src's array starts at sub_start + src*sub_stride and has sub_entries
+ *                       entries: the start position (in src's send buffer) of every sub-bag, from
+ *                       which bag boundaries are rebuilt.  Table-wise (sub_bag_major = 0): ordered
+ *                       (dst, table, sample) plus one terminal entry; the length of a sub-bag is the
+ *                       difference to the next entry.  Row-wise (sub_bag_major = 1): ordered
+ *                       (table, sample, dst) plus P terminal entries (one per dst); the length of
+ *                       sub-bag (t, s, dst) is entry[(t*b+s+1)*P + dst] - entry[(t*b+s)*P + dst]
  *   out                 fp32 [P][b][T][dim], the requester layout */
 typedef struct {
     const int32_t *sendcounts, *sdispls, *recvcounts, *rdispls;
@@ -85,6 +88,8 @@ typedef struct {
     const int32_t *sub_start;
     int64_t sub_stride;
     int64_t subbags_per_rank;
+    int64_t sub_entries;
+    int32_t sub_bag_major;
     const float *out;
 } bls_route_view_t;
 

@@ -41,7 +41,7 @@ class _View(C.Structure):
     _fields_ = [("sendcounts", C.c_void_p), ("sdispls", C.c_void_p), ("recvcounts", C.c_void_p),
                 ("rdispls", C.c_void_p), ("sendbuf", C.c_void_p), ("sendbuf_stride", C.c_int64),
                 ("sub_start", C.c_void_p), ("sub_stride", C.c_int64), ("subbags_per_rank", C.c_int64),
-                ("out", C.c_void_p)]
+                ("sub_entries", C.c_int64), ("sub_bag_major", C.c_int32), ("out", C.c_void_p)]
 
 
 _lib = None
@@ -182,7 +182,8 @@ def bls_view(plan: Plan, it: int) -> dict:
     d = {k: plan._wrap(getattr(v, k), P * P, i32).view(P, P)
          for k in ("sendcounts", "sdispls", "recvcounts", "rdispls")}
     d["sendbuf"] = plan._wrap(v.sendbuf, P * v.sendbuf_stride, i32).view(P, v.sendbuf_stride)
-    d["sub_start"] = plan._wrap(v.sub_start, P * v.sub_stride, i32).view(P, v.sub_stride)[:, :v.subbags_per_rank + 1]
+    d["sub_start"] = plan._wrap(v.sub_start, P * v.sub_stride, i32).view(P, v.sub_stride)[:, :v.sub_entries]
+    d["sub_bag_major"] = bool(v.sub_bag_major)
     d["out"] = plan.out_tensor(v.out)
     return d
 

@@ -50,7 +50,8 @@ void fill_params(BlsParams &p, const bls_table_t *tables, int T, int part, int P
     p.cap = (int)((cap + 3) / 4 * 4);          // every rank's send buffer starts on a 16-byte boundary
     p.tiles_per_table = (b + BLS_ROUTE_TB - 1) / BLS_ROUTE_TB;
     p.NT = T * p.tiles_per_table;
-    p.sub_stride = (long long)align_up((size_t)p.NQ + 1, 4);
+    // table-wise: NQ starts + 1 terminal entry; row-wise (bag-major): NQ starts + P terminal entries
+    p.sub_stride = (long long)align_up((size_t)p.NQ + (part == BLS_PART_TABLE_RR ? 1 : P), 4);
     p.out_slot_elems = (long long)P * b * T * p.D;
 }
 
@@ -142,7 +143,7 @@ bls_status_t bls_plan(const bls_table_t *tables, int T, int part, int P, int loc
     pl->routed_only = -1;
     pl->bytes = L.total;
     {   // runs of about 320 rows: long enough to amortise the start of a run, short enough to balance
-        double avg = (double)max_ids_per_rank / ((double)p.NI * local_batch);
+        double avg = (double)max_ids_per_rank / ((double)(part == BLS_PART_TABLE_RR ? p.NI : T) * local_batch);
         int R = (int)(320.0 / (avg < 0.5 ? 0.5 : avg) + 0.5);
         pl->bags_per_run = R < 4 ? 4 : (R > 64 ? 64 : R);
         pl->rows_in_flight = 4;
@@ -402,6 +403,8 @@ bls_status_t bls_view(bls_plan_t *pl, int64_t iter, bls_route_view_t *v)
     v->sub_start = p.sub_start + slot * p.P * (size_t)p.sub_stride;
     v->sub_stride = p.sub_stride;
     v->subbags_per_rank = p.NQ;
+    v->sub_entries = p.NQ + (p.part == BLS_PART_TABLE_RR ? 1 : p.P);
+    v->sub_bag_major = p.part == BLS_PART_TABLE_RR ? 0 : 1;
     v->out = p.out + slot * (size_t)p.out_slot_elems;
     return BLS_OK;
 }

@@ -67,27 +67,14 @@ template <> struct Acc<BLS_F16> {
     __device__ __forceinline__ float4 hi() const { return make_float4(c.x, c.y, d.x, d.y); }
 };
 
-__device__ __forceinline__ void red_add_v4(float *addr, float4 v)
+template <int DT>
+__device__ __forceinline__ void flush(float *o, const Acc<DT> &acc)
 {
-    asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(addr), "f"(v.x), "f"(v.y), "f"(v.z),
-                 "f"(v.w)
-                 : "memory");
+    __stcs(reinterpret_cast<float4 *>(o), acc.lo());
+    if (Acc<DT>::N == 8) __stcs(reinterpret_cast<float4 *>(o) + 1, acc.hi());
 }
 
-template <int DT, bool ROWWISE>
-__device__ __forceinline__ void flush(float *o, const Acc<DT> &acc, bool nonempty)
-{
-    if (ROWWISE) {
-        if (!nonempty) return;                         // nothing to add to the requester's sum
-        red_add_v4(o, acc.lo());
-        if (Acc<DT>::N == 8) red_add_v4(o + 4, acc.hi());
-    } else {
-        __stcs(reinterpret_cast<float4 *>(o), acc.lo());
-        if (Acc<DT>::N == 8) __stcs(reinterpret_cast<float4 *>(o) + 1, acc.hi());
-    }
-}
-
-template <int LANES, int DT, bool ROWWISE, int U>
+template <int LANES, int DT, int U>
 __global__ void __launch_bounds__(256, (U >= 8 ? 2 : 3))
 bls_gather_pool_kernel(BlsParams p, int R, int runs_per_chunk, int n_runs)
 {
@@ -166,7 +153,7 @@ bls_gather_pool_kernel(BlsParams p, int R, int runs_per_chunk, int n_runs)
                         const int y = k * U + u;
                         while (y == e_cur) {           // bags that end here (possibly empty ones)
                             if (cur >= 0) {
-                                flush<DT, ROWWISE>(o, acc, y > start);
+                                flush<DT>(o, acc);
                                 o += bag_stride;
                             }
                             acc.zero();
@@ -198,11 +185,107 @@ bls_gather_pool_kernel(BlsParams p, int R, int runs_per_chunk, int n_runs)
                 // boundary, and everything when the run has no rows at all
                 if (cur < 0) { cur = 0; start = yend; acc.zero(); }
                 for (; cur < nb; cur++) {
-                    flush<DT, ROWWISE>(o, acc, yend > start);
+                    flush<DT>(o, acc);
                     o += bag_stride;
                     acc.zero();
                     start = yend;
                 }
+            }
+        }
+        __syncwarp();
+        base = __shfl_sync(0xffffffffu, next_base, 0);
+    }
+}
+
+// Row-wise placement: the IDs of one bag are spread over the owners' regions of the
+// requester's send buffer, a handful per owner.  One lane group takes a bag, walks
+// the owners in rank order (their sub-bag starts are stored bag-major, so the P
+// starts and P ends of a bag are two contiguous reads), gathers every owner's rows
+// and keeps one running fp32 sum: the owners' partial sums are combined in owner
+// order inside registers and the pooled vector is stored once.  No atomics, no
+// zero-filled output, and the result does not depend on timing.
+template <int LANES, int DT>
+__global__ void __launch_bounds__(256, 3)
+bls_gather_rowwise_kernel(BlsParams p, int R, int runs_per_chunk, int n_runs)
+{
+    constexpr int GPW = 32 / LANES;
+    constexpr int U = LANES < 8 ? LANES : 8;
+    const int lane = threadIdx.x % LANES;
+    const int g = (threadIdx.x & 31) / LANES;
+    const unsigned gmask = LANES == 32 ? 0xffffffffu : (((1u << LANES) - 1u) << (g * LANES));
+    BlsDev *dev = p.dev;
+
+    int base = 0;
+    if ((threadIdx.x & 31) == 0) base = atomicAdd(&dev->work_ctr, GPW);
+    base = __shfl_sync(0xffffffffu, base, 0);
+    while (base < n_runs) {
+        int next_base = 0;
+        if ((threadIdx.x & 31) == 0) next_base = atomicAdd(&dev->work_ctr, GPW);
+        const int run = base + g;
+        const long long j = dev->serve_iter[0];        // row-wise: all owners answer the same iteration
+        if (run < n_runs && j >= 0) {
+            const int chunk = run / runs_per_chunk;    // (table, requester), table-major
+            const int s0 = (run - chunk * runs_per_chunk) * R;
+            const int t = chunk / p.P, src = chunk - t * p.P;
+            const int slot = (int)(j % p.S);
+            const int nb = min(R, p.b - s0);
+            const BlsTableDesc tb = p.tab[t];
+            const uint4 *rowbase = reinterpret_cast<const uint4 *>(tb.weight) + lane;
+            const unsigned rows_m1 = (unsigned)tb.rows - 1u;
+            const int *sb = p.sendbuf + ((size_t)slot * p.P + src) * (size_t)p.cap;
+            const int *ss = p.sub_start + ((size_t)slot * p.P + src) * (size_t)p.sub_stride +
+                            ((size_t)t * p.b + s0) * p.P;
+            float *o = p.out + (size_t)slot * p.out_slot_elems +
+                       (((size_t)src * p.b + s0) * p.T + t) * p.D + lane * Acc<DT>::N;
+            for (int bag = 0; bag < nb; bag++, ss += p.P, o += (size_t)p.T * p.D) {
+                Acc<DT> acc;
+                acc.zero();
+                for (int c0 = 0; c0 < p.P; c0 += LANES) {      // owners c0 .. c0+LANES-1, one per lane
+                    const int d = c0 + lane;
+                    int st = 0, en = 0;
+                    if (d < p.P) {
+                        st = min(max(ss[d], 0), p.cap);
+                        en = min(max(ss[p.P + d], st), p.cap);
+                    }
+                    const int n = en - st;
+                    int incl = n;                               // inclusive scan over the group's lanes
+                    #pragma unroll
+                    for (int w = 1; w < LANES; w <<= 1) {
+                        const int y = __shfl_up_sync(gmask, incl, w, LANES);
+                        if (lane >= w) incl += y;
+                    }
+                    const int excl = incl - n;
+                    const int total = __shfl_sync(gmask, incl, LANES - 1, LANES);
+                    for (int r0 = 0; r0 < total; r0 += LANES) {
+                        const int r = r0 + lane;                // this lane fetches the ID of row r
+                        int own = 0;                            // last lane whose first row is <= r
+                        #pragma unroll
+                        for (int step = LANES / 2; step >= 1; step >>= 1) {
+                            const int ex = __shfl_sync(gmask, excl, own + step, LANES);
+                            if (ex <= r) own += step;
+                        }
+                        const int pos = __shfl_sync(gmask, st, own, LANES) + r - __shfl_sync(gmask, excl, own, LANES);
+                        unsigned grow = 0;
+                        if (r < total) {
+                            const unsigned id = (unsigned)__ldcs(sb + pos);
+                            grow = min((unsigned)(c0 + own) * (unsigned)tb.blk + id, rows_m1);
+                        }
+                        const int m = min(LANES, total - r0);
+                        #pragma unroll 1
+                        for (int u0 = 0; u0 < m; u0 += U) {
+                            uint4 v[U];
+                            #pragma unroll
+                            for (int u = 0; u < U; u++) {
+                                const unsigned row = __shfl_sync(gmask, grow, u0 + u, LANES);
+                                v[u] = (u0 + u < m) ? __ldg(rowbase + (size_t)row * LANES) : make_uint4(0u, 0u, 0u, 0u);
+                            }
+                            #pragma unroll
+                            for (int u = 0; u < U; u++)
+                                if (u0 + u < m) acc.add(v[u]);
+                        }
+                    }
+                }
+                flush<DT>(o, acc);
             }
         }
         __syncwarp();
@@ -216,14 +299,16 @@ static void launch_gather(const bls_plan_t *pl)
     const BlsParams &p = pl->prm;
     const int R = pl->bags_per_run;
     const int rpc = (p.b + R - 1) / R;
-    const long long n_runs = (long long)p.NI * p.P * rpc;
+    const bool rowwise = p.part == BLS_PART_ROW_BLOCK;
+    // table-wise: runs of sub-bags of one (owner, table, requester); row-wise: runs of bags of one (table, requester)
+    const long long n_runs = (long long)(rowwise ? p.T : p.NI) * p.P * rpc;
     // more blocks than fit at once (late ones find the counter exhausted), fewer for small workloads
     const long long want = (n_runs + 8 * (32 / LANES) - 1) / (8 * (32 / LANES));
     const int blocks = (int)(want < 1 ? 1 : (want > pl->sm_count * 8 ? pl->sm_count * 8 : want));
-    if (p.part == BLS_PART_ROW_BLOCK)
-        bls_gather_pool_kernel<LANES, DT, true, U><<<blocks, 256, 0, pl->stream>>>(p, R, rpc, (int)n_runs);
+    if (rowwise)
+        bls_gather_rowwise_kernel<LANES, DT><<<blocks, 256, 0, pl->stream>>>(p, R, rpc, (int)n_runs);
     else
-        bls_gather_pool_kernel<LANES, DT, false, U><<<blocks, 256, 0, pl->stream>>>(p, R, rpc, (int)n_runs);
+        bls_gather_pool_kernel<LANES, DT, U><<<blocks, 256, 0, pl->stream>>>(p, R, rpc, (int)n_runs);
 }
 
 template <int LANES, int DT>

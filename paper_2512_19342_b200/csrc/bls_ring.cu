@@ -96,6 +96,12 @@ __global__ void __launch_bounds__(32) bls_gate_kernel(BlsParams p, int mode, lon
 
     // serve: all P sources (self included) have posted the iteration
     bool go_s = act && mode != BLS_MODE_ROUTE_ONLY && served < min_posted2 && is_ready;
+    if (p.part == BLS_PART_ROW_BLOCK) {
+        // row-wise: a bag needs all owners' partial sums at once, so the owners answer an
+        // iteration together, when all of them are free to act
+        const bool all_ready = __all_sync(0xffffffffu, !act || is_ready);
+        go_s = go_s && all_ready;
+    }
     long long served2 = act ? served + (go_s ? 1 : 0) : BIG;
     const long long min_served2 = warp_min_ll(served2);
 

@@ -204,18 +204,16 @@ __global__ void __launch_bounds__(1024) bls_rw_scan_kernel(BlsParams p)
         int d = threadIdx.x;
         long long end = d + 1 < p.P ? c.sdispls[d + 1] : s_total;
         c.sendcounts[d] = (int)(end - c.sdispls[d]);
+        // sub-bag starts are kept bag-major [table][sample][dst]: the entry after the last bag
+        // closes every destination's region
+        c.sub_start[(size_t)p.T * p.b * p.P + d] = (int)(end > p.cap ? p.cap : end);
     }
-    if (threadIdx.x == 0) {
-        if (s_total > p.cap) flag(p, BLS_ST_ENOSPC);
-        c.sub_start[p.NQ] = (int)(s_total > p.cap ? p.cap : s_total);
-    }
+    if (threadIdx.x == 0 && s_total > p.cap) flag(p, BLS_ST_ENOSPC);
 }
 
 // grid (NT, P), one thread per bag.  Inside a tile, the lookups of one
 // destination keep their original order: position = tile base + number of
 // same-destination lookups in earlier bags of the tile + rank inside the bag.
-// Also clears the tile's part of the requester's output slot, into which the
-// owners will add their partial sums.
 __global__ void __launch_bounds__(BLS_ROUTE_TB) bls_rw_scatter_kernel(BlsParams p)
 {
     __shared__ int cnt[BLS_MAX_RANKS][BLS_ROUTE_TB + 1];
@@ -260,7 +258,7 @@ __global__ void __launch_bounds__(BLS_ROUTE_TB) bls_rw_scatter_kernel(BlsParams 
     if (s < nb) {
         for (int d = 0; d < p.P; d++) {
             int pos = cnt[d][s];
-            c.sub_start[((size_t)d * p.T + t) * p.b + s0 + s] = pos > p.cap ? p.cap : pos;
+            c.sub_start[((size_t)t * p.b + s0 + s) * p.P + d] = pos > p.cap ? p.cap : pos;
         }
         for (int l = st; l < en; l++) {
             int id = c.ids[l];
@@ -269,14 +267,6 @@ __global__ void __launch_bounds__(BLS_ROUTE_TB) bls_rw_scatter_kernel(BlsParams 
             int pos = cnt[d][s]++;
             if (pos < p.cap) c.sendbuf[pos] = id - d * blk;
         }
-    }
-    // clear out[slot][src][s0 .. s0+nb)[t][:]
-    float4 *out = reinterpret_cast<float4 *>(p.out + (size_t)c.slot * p.out_slot_elems);
-    const int d4 = p.D / 4;
-    for (int e = threadIdx.x; e < nb * d4; e += blockDim.x) {
-        int bag = e / d4, col = e % d4;
-        size_t idx = ((((size_t)src * p.b + s0 + bag) * p.T + t) * p.D) / 4 + col;
-        out[idx] = make_float4(0.f, 0.f, 0.f, 0.f);
     }
 }
 

@@ -51,7 +51,8 @@ def check_route(w, view, ids, off):
     for src in range(P):
         n = int(base[src + 1] - base[src])
         assert np.array_equal(sendbuf[src, :n], art["sendbuf"][base[src]:base[src + 1]]), f"sendbuf of rank {src}"
-        assert sub[src, -1] == n and sub[src, 0] == 0
+        if not view["sub_bag_major"]:
+            assert sub[src, -1] == n and sub[src, 0] == 0
         for d in range(P):
             lo = art["sdispls"][src, d]
             recv_parts[(d, src)] = sendbuf[src, lo:lo + art["sendcounts"][src, d]]
@@ -59,13 +60,22 @@ def check_route(w, view, ids, off):
     recv = np.concatenate([recv_parts[(d, s)] for d in range(P) for s in range(P)]) if len(ids) else np.zeros(0, np.int32)
     assert np.array_equal(recv, art["recvbuf"])
     # sub-bag lengths in (dst, src, bag) order
-    lens = np.diff(sub.astype(np.int64), axis=1)
     got, pos = [], 0
-    for d in range(P):
-        per = oracle.subbags_per_pair(w.partition, P, T, b, d)
-        for src in range(P):
-            got.append(lens[src, pos:pos + per])
-        pos += per
+    if view["sub_bag_major"]:                      # row-wise: entries ordered (table, sample, dst)
+        s3 = sub.astype(np.int64).reshape(P, T * b + 1, P)
+        assert np.array_equal(s3[:, 0, :], art["sdispls"])
+        assert np.array_equal(s3[:, -1, :], art["sdispls"] + art["sendcounts"])
+        lens3 = np.diff(s3, axis=1)                # [src][bag][dst]
+        for d in range(P):
+            for src in range(P):
+                got.append(lens3[src, :, d])
+    else:
+        lens = np.diff(sub.astype(np.int64), axis=1)
+        for d in range(P):
+            per = oracle.subbags_per_pair(w.partition, P, T, b, d)
+            for src in range(P):
+                got.append(lens[src, pos:pos + per])
+            pos += per
     assert np.array_equal(np.concatenate(got), art["sublen"])
     return art
 
