@@ -1,0 +1,70 @@
+"""Full-size workloads 3, 4 and 5 in the configuration the benchmark times
+(hash-filled tables, bls_step with the workload's largest bound, then the drain).
+
+Routing artefacts of a whole iteration are compared with the oracle bit for
+bit; pooled vectors are compared on sampled bags that the oracle evaluates one
+by one from the counter-hash definition of the tables (the 33 GB and 64 GB
+tables never exist on the host).  GPU only."""
+import numpy as np
+import pytest
+import torch
+
+import bls_inputs as bi
+import oracle
+import paper_2512_19342_b200 as bls
+from test_gpu_parity import TDT, TOL, check_route
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.mark.parametrize("num", [3, 4, 5])
+def test_full_size_iteration(num):
+    w = bi.workload(num)
+    need = w.table_bytes() * 1.25 + 8e9
+    if torch.cuda.get_device_properties(0).total_memory < need:
+        pytest.skip("not enough device memory for this workload")
+    P, T, b, D = w.P, w.T, w.local_batch, w.tables[0].dim
+    tabs = []
+    for spec in w.tables:
+        t = torch.empty(spec.rows, spec.dim, dtype=TDT[spec.dtype], device="cuda")
+        bls.bls_fill_hash_table(t, spec.seed, spec.index)
+        tabs.append(t)
+    # the fill kernel against the generator, on rows spread over a table (first, last, random)
+    rng = np.random.Generator(np.random.PCG64(num))
+    spec = w.tables[T - 1]
+    pick = np.unique(np.concatenate([[0, spec.rows - 1], rng.integers(0, spec.rows, 64)]))
+    got = tabs[T - 1][torch.from_numpy(pick).cuda()].cpu()
+    want = bi.hash_rows(spec.seed, spec.index, pick, spec.dim, spec.dtype)
+    got = got.numpy() if spec.dtype == "f32" else got.view(torch.int16).numpy().view(np.uint16)
+    assert np.array_equal(got, want.view(np.uint16) if spec.dtype == "f16" else want)
+
+    ids, off = bi.make_iteration(w, 0)
+    cap = int(np.diff(off[::T * b].astype(np.int64)).max()) + 64
+    k = max(w.ks)
+    plan = bls.bls_plan(tabs, w.partition, P, b, k, cap)
+    d_ids, d_off = torch.from_numpy(ids).cuda(), torch.from_numpy(off).cuda()
+    out, it = bls.bls_step(plan, k, d_ids, d_off)
+    assert (out is None) == (k > 0)
+    view = bls.bls_view(plan, 0)
+    check_route(w, view, ids, off)                     # counts, displacements, packed buffers, sub-bag lengths
+    while True:
+        o, it = bls.bls_drain(plan)
+        if o is None:
+            break
+        out = o
+    assert bls.bls_status(plan)[0] == bls.BLS_OK
+    # sampled bags: random ones plus the longest, an empty one if any, the first and the last
+    lens = np.diff(off.astype(np.int64))
+    G = P * T * b
+    sel = set(rng.integers(0, G, 3000).tolist()) | {0, G - 1, int(lens.argmax()), int(lens.argmin())}
+    sel = np.array(sorted(sel), dtype=np.int64)
+    want = oracle.pool_definition(P, T, b, w.tables, None, ids, off, sel=sel, nthreads=8)
+    src, t, s = sel // (T * b), (sel // b) % T, sel % b
+    got = out[torch.from_numpy(src).cuda(), torch.from_numpy(s).cuda(), torch.from_numpy(t).cuda()].cpu().numpy()
+    err = oracle.vector_rel_err(got, want)
+    assert err <= TOL[w.tables[0].dtype], err
+    empty = lens[sel] == 0
+    assert np.all(got[empty] == 0)
+    # properties that hold at any size: every bag written, totals consistent
+    assert int(view["sendcounts"].sum()) == len(ids)
+    assert torch.isfinite(out).all()
