@@ -32,6 +32,7 @@ NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
 DT_BYTES = {"f32": 4, "bf16": 2, "f16": 2}
 N_DISTINCT = {1: 10, 2: 16, 3: 8, 4: 3, 5: 3}       # distinct ID batches kept resident and cycled
+HOT_DEFAULT = {}                                     # hot rows per table staged in shared memory, by workload
 
 
 def parse_args():
@@ -45,6 +46,8 @@ def parse_args():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--tables", type=int, default=0, help="keep only the first N tables (reduced profiling case)")
     ap.add_argument("--tune", default="", help="bags_per_run,rows_in_flight for the gather kernel (0 = default)")
+    ap.add_argument("--hot", type=int, default=-1,
+                    help="hot rows per table staged in shared memory (0 = off, -1 = the workload's default)")
     ap.add_argument("--ks", default="", help="comma-separated bounds to time instead of the workload's own")
     return ap.parse_args()
 
@@ -312,6 +315,17 @@ def run_mine(args):
 
     if args.tune:
         bls.bls_set_tuning(plan, *[int(x) for x in args.tune.split(",")])
+    hot_k = HOT_DEFAULT.get(args.config, 0) if args.hot < 0 else args.hot
+    if hot_k and w.partition == "table_rr":
+        # request statistics come from two batches that are not among the timed ones
+        bls.bls_hot_attach(plan, hot_k)
+        for it in (nd, nd + 1):
+            ids_l, off_l = bi.make_iteration(w, it)
+            bls.bls_hot_observe(plan, torch.from_numpy(ids_l).cuda(), torch.from_numpy(off_l).cuda())
+        bls.bls_hot_build(plan)
+        torch.cuda.synchronize()
+    else:
+        hot_k = 0
 
     def loop(k, steps):
         for t in range(steps):
@@ -398,6 +412,7 @@ def run_mine(args):
         "config": {"workload": w.name, "tables": w.T, "rows": [t.rows for t in w.tables][:3] + ["..."],
                    "dim": w.tables[0].dim, "P": w.P, "partition": w.partition, "global_batch": w.global_batch,
                    "lookups_per_step": L_mean, "k": k_head, "multi_gpu": "replicas only",
+                   "hot_rows_per_table": hot_k,
                    "l2": f"inputs larger than L2: tables {w.table_bytes() / 1e9:.2f} GB, {nd} distinct ID batches cycled"},
         "by_k": {str(k): {"lookups_per_s": t / (m * 1e-3), "ms_per_step": m / args.steps} for k, (m, t) in by_k.items()},
         "max_lag": lag,

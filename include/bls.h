@@ -176,6 +176,31 @@ bls_status_t bls_profile_read(bls_plan_t *plan, double *ms_route, double *ms_gat
  * worth), rows_in_flight = row loads per batch, 4 or 8 (0 = keep; default 4). */
 bls_status_t bls_set_tuning(bls_plan_t *plan, int bags_per_run, int rows_in_flight);
 
+/* ---- hot-row staging (optional; table-wise placement only) ----
+ * Power-law ID distributions put most lookups on a few hundred rows per table.
+ * After bls_hot_build the router marks, for every packed lookup, the slot of its
+ * row in the table's hot list, and the gather kernel keeps the listed rows of the
+ * table it is working on in shared memory.  Pooled results are unchanged (a staged
+ * row is a copy of the table row).  The paper calls caching orthogonal to its
+ * collective (Section II); this is an internal optimisation of step (2).
+ *   bls_hot_bytes    size of the caller-provided device buffer for `rows_per_table` slots
+ *   bls_hot_attach   hand over that buffer (device, 256-byte aligned, borrowed until
+ *                    bls_destroy); rows_per_table * row bytes must fit in shared memory
+ *                    (<= 200 KiB), nothing may be outstanding; synchronises the stream
+ *   bls_hot_observe  add one batch of IDs (device, same layout as bls_step's) to the
+ *                    per-row request counts; asynchronous
+ *   bls_hot_build    select per table the most requested rows (at most rows_per_table,
+ *                    cut at a count threshold) and switch staging on; asynchronous;
+ *                    nothing may be outstanding
+ *   bls_hot_view     device pointers to the lists: rows int32 [T][rows_per_table] in slot
+ *                    order, count int32 [T] */
+bls_status_t bls_hot_bytes(bls_plan_t *plan, int rows_per_table, size_t *bytes /*host*/);
+bls_status_t bls_hot_attach(bls_plan_t *plan, int rows_per_table, void *buffer, size_t bytes);
+bls_status_t bls_hot_observe(bls_plan_t *plan, const int32_t *ids, const int32_t *offsets, int64_t n_ids);
+bls_status_t bls_hot_build(bls_plan_t *plan);
+bls_status_t bls_hot_view(bls_plan_t *plan, const int32_t **rows /*host out*/, const int32_t **count /*host out*/,
+                          int *rows_per_table /*host out*/);
+
 const char *bls_strerror(int status);
 
 /* ---- input generation helper (not part of the method) ----

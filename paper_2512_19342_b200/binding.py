@@ -13,7 +13,7 @@ from typing import List, Optional, Sequence, Tuple
 import torch
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "libbls.so")
+LIB_PATH = os.environ.get("BLS_LIBRARY", os.path.join(_HERE, "libbls.so"))   # override: an alternative build
 
 BLS_OK, BLS_EINVAL, BLS_ENOSPC, BLS_ECUDA, BLS_ERANGE, BLS_ETIMEOUT, BLS_ESTATE = range(7)
 BLS_F32, BLS_BF16, BLS_F16 = 0, 1, 2
@@ -24,7 +24,8 @@ _DTYPE = {torch.float32: BLS_F32, torch.bfloat16: BLS_BF16, torch.float16: BLS_F
 EXPORTS = ["bls_plan_bytes", "bls_plan", "bls_destroy", "bls_route", "bls_lookup", "bls_step",
            "bls_drain", "bls_step_host", "bls_drain_host", "bls_view", "bls_counters", "bls_status",
            "bls_set_stall", "bls_set_wait_limit", "bls_strerror", "bls_fill_hash_table",
-           "bls_profile", "bls_profile_read", "bls_set_tuning", "bls_route_table_rr_static"]
+           "bls_profile", "bls_profile_read", "bls_set_tuning", "bls_route_table_rr_static",
+           "bls_hot_bytes", "bls_hot_attach", "bls_hot_observe", "bls_hot_build", "bls_hot_view"]
 
 
 class BlsError(RuntimeError):
@@ -250,3 +251,36 @@ def bls_route_table_rr_static(table_rows: torch.Tensor, P: int, local_batch: int
         C.c_void_p(sdispls.data_ptr()), C.c_void_p(sendbuf.data_ptr()), C.c_int64(sendbuf.shape[1]),
         C.c_void_p(sub_start.data_ptr()), C.c_void_p(status.data_ptr()), _stream_ptr(stream)),
         "bls_route_table_rr_static")
+
+
+def bls_hot_attach(plan: Plan, rows_per_table: int) -> None:
+    """Allocate (with torch) and attach the buffer for hot-row staging with `rows_per_table` slots."""
+    n = C.c_size_t(0)
+    _check(lib().bls_hot_bytes(plan.handle, rows_per_table, C.byref(n)), "bls_hot_bytes")
+    buf = torch.empty(n.value + 256, dtype=torch.uint8, device=plan.workspace.device)
+    pad = (-buf.data_ptr()) % 256
+    buf = buf[pad:pad + n.value]
+    _check(lib().bls_hot_attach(plan.handle, rows_per_table, C.c_void_p(buf.data_ptr()), C.c_size_t(n.value)),
+           "bls_hot_attach")
+    plan.hot_buffer, plan.hot_rows_per_table = buf, rows_per_table
+
+
+def bls_hot_observe(plan: Plan, ids: torch.Tensor, offsets: torch.Tensor) -> None:
+    _check(lib().bls_hot_observe(plan.handle, C.c_void_p(ids.data_ptr()), C.c_void_p(offsets.data_ptr()),
+                                 C.c_int64(ids.numel())), "bls_hot_observe")
+
+
+def bls_hot_build(plan: Plan) -> None:
+    _check(lib().bls_hot_build(plan.handle), "bls_hot_build")
+
+
+def bls_hot_view(plan: Plan):
+    """(rows [T][K] int32, count [T] int32) as views into the attached buffer."""
+    rows, count, k = C.c_void_p(), C.c_void_p(), C.c_int(0)
+    _check(lib().bls_hot_view(plan.handle, C.byref(rows), C.byref(count), C.byref(k)), "bls_hot_view")
+    buf = plan.hot_buffer
+
+    def wrap(ptr, n):
+        off = ptr - buf.data_ptr()
+        return buf[off:off + 4 * n].view(torch.int32)
+    return wrap(rows.value, plan.T * k.value).view(plan.T, k.value), wrap(count.value, plan.T)

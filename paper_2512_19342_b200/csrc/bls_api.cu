@@ -142,6 +142,9 @@ bls_status_t bls_plan(const bls_table_t *tables, int T, int part, int P, int loc
     pl->k_cur = -1;
     pl->routed_only = -1;
     pl->bytes = L.total;
+    pl->h_rows = (long long *)malloc(sizeof(long long) * T);
+    if (!pl->h_rows) { free(pl); return BLS_ENOSPC; }
+    for (int t = 0; t < T; t++) pl->h_rows[t] = tables[t].rows;
     {   // runs of about 320 rows: long enough to amortise the start of a run, short enough to balance
         double avg = (double)max_ids_per_rank / ((double)(part == BLS_PART_TABLE_RR ? p.NI : T) * local_batch);
         int R = (int)(320.0 / (avg < 0.5 ? 0.5 : avg) + 0.5);
@@ -151,6 +154,7 @@ bls_status_t bls_plan(const bls_table_t *tables, int T, int part, int P, int loc
     int devid = 0;
     if (!cuda_ok(cudaGetDevice(&devid)) ||
         !cuda_ok(cudaDeviceGetAttribute(&pl->sm_count, cudaDevAttrMultiProcessorCount, devid))) {
+        free(pl->h_rows);
         free(pl);
         return BLS_ECUDA;
     }
@@ -201,7 +205,7 @@ bls_status_t bls_plan(const bls_table_t *tables, int T, int part, int P, int loc
               cuda_ok(cudaMemsetAsync(ws + L.counts, 0, sizeof(int) * p.S * 4 * P * P, pl->stream)) &&
               // the vectors above are pageable: make sure the copies have left them
               cuda_ok(cudaStreamSynchronize(pl->stream));
-    if (!ok) { free(pl); return BLS_ECUDA; }
+    if (!ok) { free(pl->h_rows); free(pl); return BLS_ECUDA; }
     *plan = pl;
     return BLS_OK;
 }
@@ -213,6 +217,7 @@ void bls_destroy(bls_plan_t *plan)
         for (int i = 0; i < BLS_PROF_MAX * 4; i++) cudaEventDestroy(plan->prof_ev[i]);
         free(plan->prof_ev);
     }
+    free(plan->h_rows);
     free(plan);
 }
 

@@ -16,6 +16,7 @@
 // streaming loads/stores so that they do not evict table rows.
 #include <cuda_bf16.h>
 #include <cuda_fp16.h>
+#include <type_traits>
 #include "bls_internal.h"
 
 // fp32 accumulators as packed pairs: sm_100 adds two fp32 lanes per instruction
@@ -74,16 +75,131 @@ __device__ __forceinline__ void flush(float *o, const Acc<DT> &acc)
     if (Acc<DT>::N == 8) __stcs(reinterpret_cast<float4 *>(o) + 1, acc.hi());
 }
 
+// One run: nb consecutive sub-bags of pair `pr` requested by rank `src`, starting at
+// sample s0, in ring slot `slot`.  With HOT, lookups whose slot number (written by
+// the router) is below K read their row from the staged copy in shared memory.
+template <int LANES, int DT, int U, bool HOT>
+__device__ __forceinline__ void stream_run(const BlsParams &p, const BlsPairDesc &pr, int i, int slot, int src,
+                                           int s0, int nb, int lane, const uint4 *hot_rows)
+{
+    constexpr int Q = U / 4;                           // 16-byte ID quads per batch
+    const size_t bag_stride = (size_t)p.T * p.D;       // floats between consecutive samples in out
+    const int *ss = p.sub_start + ((size_t)slot * p.P + src) * (size_t)p.sub_stride + (size_t)i * p.b + s0;
+    const int p0 = min(max(ss[0], 0), p.cap);
+    const int n = min(max(ss[nb], p0), p.cap) - p0;    // rows in this run
+    // The ID stream is read in aligned 16-byte quads and processed in whole batches
+    // of U rows: stream coordinate y = a + x, where x counts the run's rows and
+    // a = p0 mod 4.  The a IDs before the run and the IDs after it up to the end of
+    // the last batch belong to other bags (or to nobody); their rows are loaded
+    // (clamped, so always in bounds) and accumulated into a "bag" that is never
+    // stored.  That keeps the inner loop free of validity predicates.
+    const int a = p0 & 3;
+    const int yend = a + n;
+    const int org = a - p0;                            // y coordinate of send-buffer position 0
+    // bag c of the run ends at bag_end(c); c = -1 is the part before the run, c = nb the part after
+    auto bag_end = [&](int c) {
+        return c < 0 ? a : c < nb - 1 ? min(max(ss[c + 1] + org, a), yend) : c == nb - 1 ? yend : 0x7fffffff;
+    };
+    int cur = -1;
+    int e_cur = a, e_nxt = bag_end(0);
+    const size_t row0 = ((size_t)slot * p.P + src) * (size_t)p.cap + (p0 - a);
+    const int4 *sq = reinterpret_cast<const int4 *>(p.sendbuf + row0);
+    const uint2 *hq = HOT ? reinterpret_cast<const uint2 *>(p.hot.hotslot + row0) : nullptr;
+    const uint4 *rowbase = reinterpret_cast<const uint4 *>(pr.base) + lane;
+    const unsigned nrows_m1 = (unsigned)pr.nrows - 1u;
+    const unsigned K = HOT ? (unsigned)p.hot.K : 0u;
+    float *o = p.out + (size_t)slot * p.out_slot_elems +
+               (((size_t)src * p.b + s0) * p.T + pr.t) * p.D + lane * Acc<DT>::N;
+
+    Acc<DT> acc;
+    acc.zero();
+    int4 ida[Q], idb[Q];                               // IDs of the next batch for va / for vb
+    uint2 ha[Q], hb[Q];                                // and their staged-copy slots
+    uint4 va[U], vb[U];
+    const int nbat = (yend + U - 1) / U;
+
+    auto load_ids = [&](int4(&idq)[Q], uint2(&hsq)[Q], int k) {
+        if (k >= nbat) return;
+        #pragma unroll
+        for (int q = 0; q < Q; q++) {
+            idq[q] = __ldcs(sq + k * Q + q);
+            if (HOT) hsq[q] = __ldcs(hq + k * Q + q);
+        }
+    };
+    auto issue = [&](uint4(&v)[U], const int4(&idq)[Q], const uint2(&hsq)[Q], int k) {
+        if (k >= nbat) return;
+        #pragma unroll
+        for (int u = 0; u < U; u++) {
+            const unsigned id = (unsigned)(&idq[u / 4].x)[u & 3];
+            if constexpr (HOT) {
+                const unsigned w = (&hsq[u / 4].x)[(u & 3) >> 1];
+                const unsigned hs = (u & 1) ? (w >> 16) : (w & 0xffffu);
+                // one generic load, no branch: the address is in shared memory for a staged row,
+                // in the table otherwise (lane groups of a warp differ, a branch would diverge)
+                const uint4 *src_row = hs < K ? hot_rows + hs * LANES + lane : rowbase + (size_t)min(id, nrows_m1) * LANES;
+                v[u] = *src_row;
+            } else {
+                v[u] = __ldg(rowbase + (size_t)min(id, nrows_m1) * LANES);
+            }
+        }
+    };
+    auto consume = [&](const uint4(&v)[U], int k) {
+        if (k >= nbat) return;
+        if (e_cur >= k * U + U) {                      // no bag ends inside this batch
+            #pragma unroll
+            for (int u = 0; u < U; u++) acc.add(v[u]);
+            return;
+        }
+        #pragma unroll
+        for (int u = 0; u < U; u++) {
+            const int y = k * U + u;
+            while (y == e_cur) {                       // bags that end here (possibly empty ones)
+                if (cur >= 0) {
+                    flush<DT>(o, acc);
+                    o += bag_stride;
+                }
+                acc.zero();
+                cur++;
+                e_cur = e_nxt;
+                e_nxt = bag_end(cur + 1);
+            }
+            acc.add(v[u]);
+        }
+    };
+
+    // Pipeline: the IDs of a batch are fetched two batches before its rows are
+    // requested, and its rows one batch before they are added, so that neither the ID
+    // latency nor the row latency sits on the critical path.
+    load_ids(ida, ha, 0);
+    load_ids(idb, hb, 1);
+    issue(va, ida, ha, 0);
+    load_ids(ida, ha, 2);
+    for (int k = 0; k < nbat; k += 2) {
+        issue(vb, idb, hb, k + 1);
+        load_ids(idb, hb, k + 3);
+        consume(va, k);
+        issue(va, ida, ha, k + 2);
+        load_ids(ida, ha, k + 4);
+        consume(vb, k + 1);
+    }
+    // bags not closed by a row after them: the last one when the run ends on a batch
+    // boundary, and everything when the run has no rows at all
+    if (cur < 0) { cur = 0; acc.zero(); }
+    for (; cur < nb; cur++) {
+        flush<DT>(o, acc);
+        o += bag_stride;
+        acc.zero();
+    }
+}
+
 template <int LANES, int DT, int U>
 __global__ void __launch_bounds__(256, (U >= 8 ? 2 : 3))
 bls_gather_pool_kernel(BlsParams p, int R, int runs_per_chunk, int n_runs)
 {
     constexpr int GPW = 32 / LANES;                    // groups (runs) per warp
-    constexpr int Q = U / 4;                           // 16-byte ID quads per batch
     const int lane = threadIdx.x % LANES;
     const int g = (threadIdx.x & 31) / LANES;
     BlsDev *dev = p.dev;
-    const size_t bag_stride = (size_t)p.T * p.D;       // floats between consecutive samples in out
 
     int base = 0;
     if ((threadIdx.x & 31) == 0) base = atomicAdd(&dev->work_ctr, GPW);
@@ -98,102 +214,89 @@ bls_gather_pool_kernel(BlsParams p, int R, int runs_per_chunk, int n_runs)
             const int i = chunk / p.P, src = chunk - i * p.P;
             const BlsPairDesc pr = p.pair[i];
             const long long j = dev->serve_iter[pr.dst];
-            if (j >= 0) {                              // else: this owner does not serve in this wave
-                const int slot = (int)(j % p.S);
-                const int nb = min(R, p.b - s0);
-                const int *ss = p.sub_start + ((size_t)slot * p.P + src) * (size_t)p.sub_stride + (size_t)i * p.b + s0;
-                const int p0 = min(max(ss[0], 0), p.cap);
-                const int n = min(max(ss[nb], p0), p.cap) - p0;          // rows in this run
-                // The ID stream is read in aligned 16-byte quads and processed in whole batches
-                // of U rows: stream coordinate y = a + x, where x counts the run's rows and
-                // a = p0 mod 4.  The a IDs before the run and the IDs after it up to the end of
-                // the last batch belong to other bags (or to nobody); their rows are loaded
-                // (clamped, so always in bounds) and accumulated into a "bag" that is never
-                // stored.  That keeps the inner loop free of validity predicates.
-                const int a = p0 & 3;
-                const int yend = a + n;
-                const int org = a - p0;                // y coordinate of send-buffer position 0
-                // bag c of the run ends at bag_end(c); c = -1 is the part before the run, c = nb the part after
-                auto bag_end = [&](int c) {
-                    return c < 0 ? a : c < nb - 1 ? min(max(ss[c + 1] + org, a), yend) : c == nb - 1 ? yend : 0x7fffffff;
-                };
-                int cur = -1;
-                int e_cur = a, e_nxt = bag_end(0);
-                int start = 0;                         // y where the current bag started
-                const int4 *sq = reinterpret_cast<const int4 *>(
-                    p.sendbuf + ((size_t)slot * p.P + src) * (size_t)p.cap + (p0 - a));
-                const uint4 *rowbase = reinterpret_cast<const uint4 *>(pr.base) + lane;
-                const unsigned nrows_m1 = (unsigned)pr.nrows - 1u;
-                float *o = p.out + (size_t)slot * p.out_slot_elems +
-                           (((size_t)src * p.b + s0) * p.T + pr.t) * p.D + lane * Acc<DT>::N;
-
-                Acc<DT> acc;
-                acc.zero();
-                int4 ida[Q], idb[Q];                   // IDs of the next batch for va / for vb
-                uint4 va[U], vb[U];
-                const int nbat = (yend + U - 1) / U;
-
-                auto load_ids = [&](int4(&idq)[Q], int k) {
-                    if (k >= nbat) return;
-                    #pragma unroll
-                    for (int q = 0; q < Q; q++) idq[q] = __ldcs(sq + k * Q + q);
-                };
-                auto issue = [&](uint4(&v)[U], const int4(&idq)[Q], int k) {
-                    if (k >= nbat) return;
-                    #pragma unroll
-                    for (int u = 0; u < U; u++) {
-                        const unsigned id = (unsigned)(&idq[u / 4].x)[u & 3];
-                        v[u] = __ldg(rowbase + (size_t)min(id, nrows_m1) * LANES);
-                    }
-                };
-                auto consume = [&](const uint4(&v)[U], int k) {
-                    if (k >= nbat) return;
-                    #pragma unroll
-                    for (int u = 0; u < U; u++) {
-                        const int y = k * U + u;
-                        while (y == e_cur) {           // bags that end here (possibly empty ones)
-                            if (cur >= 0) {
-                                flush<DT>(o, acc);
-                                o += bag_stride;
-                            }
-                            acc.zero();
-                            cur++;
-                            start = y;
-                            e_cur = e_nxt;
-                            e_nxt = bag_end(cur + 1);
-                        }
-                        acc.add(v[u]);
-                    }
-                };
-
-                // Pipeline: the IDs of a batch are fetched two batches before its rows are
-                // requested, and its rows one batch before they are added, so that neither the ID
-                // latency nor the row latency sits on the critical path.
-                load_ids(ida, 0);
-                load_ids(idb, 1);
-                issue(va, ida, 0);
-                load_ids(ida, 2);
-                for (int k = 0; k < nbat; k += 2) {
-                    issue(vb, idb, k + 1);
-                    load_ids(idb, k + 3);
-                    consume(va, k);
-                    issue(va, ida, k + 2);
-                    load_ids(ida, k + 4);
-                    consume(vb, k + 1);
-                }
-                // bags not closed by a row after them: the last one when the run ends on a batch
-                // boundary, and everything when the run has no rows at all
-                if (cur < 0) { cur = 0; start = yend; acc.zero(); }
-                for (; cur < nb; cur++) {
-                    flush<DT>(o, acc);
-                    o += bag_stride;
-                    acc.zero();
-                    start = yend;
-                }
-            }
+            if (j >= 0)                                // else: this owner does not serve in this wave
+                stream_run<LANES, DT, U, false>(p, pr, i, (int)(j % p.S), src, s0, min(R, p.b - s0), lane, nullptr);
         }
         __syncwarp();
         base = __shfl_sync(0xffffffffu, next_base, 0);
+    }
+}
+
+// Hot-row variant: one persistent block per SM.  Blocks start spread over the
+// (owner, table) pairs; a block copies its pair's hot rows into shared memory once
+// and takes runs from the pair's counter until the pair is used up.  After that its
+// warps help with whatever the other pairs have left, without staging (leftovers
+// are small, and a fresh copy would cost more than it saves).
+template <int LANES, int DT>
+__global__ void __launch_bounds__(768, 1)
+bls_gather_hot_kernel(BlsParams p, int R, int runs_per_chunk)
+{
+    extern __shared__ uint4 hot_rows[];                // [K][LANES]
+    constexpr int GPW = 32 / LANES;
+    const int lane = threadIdx.x % LANES;
+    const int wl = threadIdx.x & 31;
+    const int g = wl / LANES;
+    BlsDev *dev = p.dev;
+    const int runs_in_pair = p.P * runs_per_chunk;
+    const int i0 = (int)(((long long)blockIdx.x * p.NI) / gridDim.x);
+
+    auto take_runs = [&](int i, auto hot_tag) {        // all runs this warp can get from pair i
+        constexpr bool HOT = decltype(hot_tag)::value;
+        const BlsPairDesc pr = p.pair[i];
+        const long long j = dev->serve_iter[pr.dst];
+        if (j < 0) return;                             // this owner does not serve in this wave
+        int base = 0;
+        if (wl == 0) base = atomicAdd(&p.hot.pair_ctr[i], GPW);
+        base = __shfl_sync(0xffffffffu, base, 0);
+        while (base < runs_in_pair) {
+            int next_base = 0;
+            if (wl == 0) next_base = atomicAdd(&p.hot.pair_ctr[i], GPW);
+            const int run = base + g;
+            if (run < runs_in_pair) {
+                const int src = run / runs_per_chunk;
+                const int s0 = (run - src * runs_per_chunk) * R;
+                stream_run<LANES, DT, 4, HOT>(p, pr, i, (int)(j % p.S), src, s0, min(R, p.b - s0), lane, hot_rows);
+            }
+            __syncwarp();
+            base = __shfl_sync(0xffffffffu, next_base, 0);
+        }
+    };
+
+    {   // stage the hot rows of the block's own pair: eight independent loads per thread at a time
+        const BlsPairDesc pr = p.pair[i0];
+        const int tot = min(p.hot.count[pr.t], p.hot.K) * LANES;
+        const int *list = p.hot.rows + (size_t)pr.t * p.hot.K;
+        const uint4 *tbl = reinterpret_cast<const uint4 *>(pr.base);
+        for (int e0 = 0; e0 < tot; e0 += 8 * blockDim.x) {
+            uint4 tmp[8];
+            #pragma unroll
+            for (int k = 0; k < 8; k++) {
+                const int e = e0 + k * blockDim.x + threadIdx.x;
+                if (e < tot) {
+                    const unsigned row = min((unsigned)list[e / LANES], (unsigned)pr.nrows - 1u);
+                    tmp[k] = __ldg(tbl + (size_t)row * LANES + (e % LANES));
+                }
+            }
+            #pragma unroll
+            for (int k = 0; k < 8; k++) {
+                const int e = e0 + k * blockDim.x + threadIdx.x;
+                if (e < tot) hot_rows[e] = tmp[k];
+            }
+        }
+    }
+    __syncthreads();
+    take_runs(i0, std::true_type{});
+    // leftovers of the other pairs: each lane looks at one pair's counter, the warp visits those with work
+    for (int q0 = 1; q0 < p.NI; q0 += 32) {
+        const int q = q0 + wl;
+        bool has = false;
+        if (q < p.NI) has = *(volatile int *)&p.hot.pair_ctr[(i0 + q) % p.NI] < runs_in_pair;
+        unsigned m = __ballot_sync(0xffffffffu, has);
+        while (m) {
+            const int b = __ffs(m) - 1;
+            m &= m - 1;
+            take_runs((i0 + q0 + b) % p.NI, std::false_type{});
+        }
     }
 }
 
@@ -305,9 +408,20 @@ static void launch_gather(const bls_plan_t *pl)
     // more blocks than fit at once (late ones find the counter exhausted), fewer for small workloads
     const long long want = (n_runs + 8 * (32 / LANES) - 1) / (8 * (32 / LANES));
     const int blocks = (int)(want < 1 ? 1 : (want > pl->sm_count * 8 ? pl->sm_count * 8 : want));
-    if (rowwise)
+    if (rowwise) {
         bls_gather_rowwise_kernel<LANES, DT><<<blocks, 256, 0, pl->stream>>>(p, R, rpc, (int)n_runs);
-    else
+    } else if (p.hot.enabled) {
+        const size_t smem = (size_t)p.hot.K * p.row_bytes;
+        static size_t configured = 0;                  // per instantiation: shared memory size it was set up for
+        if (configured != smem) {
+            cudaFuncSetAttribute(bls_gather_hot_kernel<LANES, DT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+            // leave the rest of the SM's on-chip memory to L1
+            int pct = (int)((smem + 2048) * 100 / (228 * 1024)) + 1;
+            cudaFuncSetAttribute(bls_gather_hot_kernel<LANES, DT>, cudaFuncAttributePreferredSharedMemoryCarveout, pct > 100 ? 100 : pct);
+            configured = smem;
+        }
+        bls_gather_hot_kernel<LANES, DT><<<pl->sm_count, 768, smem, pl->stream>>>(p, R, rpc);
+    } else
         bls_gather_pool_kernel<LANES, DT, U><<<blocks, 256, 0, pl->stream>>>(p, R, rpc, (int)n_runs);
 }
 

@@ -54,6 +54,23 @@ struct BlsPairDesc {
     int pad;
 };
 
+// Hot-row staging (optional, table-wise placement): per table the K most frequently
+// requested rows, found from observed ID batches, are copied into shared memory by
+// the gather kernel; the router marks every lookup with its slot in that copy.
+struct BlsHot {
+    int enabled;                 // lists built: the router marks lookups, the gather kernel stages rows
+    int K;                       // slots per table
+    unsigned *counts;            // [sum rows]    observed request counts
+    unsigned *bitmap;            // [sum words]   bit r of table t set: row r is hot
+    unsigned *prefix;            // [sum words]   hot rows of the table before this word
+    const long long *row_base;   // [T+1] first counter of table t
+    const long long *word_base;  // [T+1] first bitmap word of table t
+    int *rows;                   // [T][K] hot row numbers, slot order
+    int *count;                  // [T]    hot rows of table t (<= K)
+    unsigned short *hotslot;     // [S][P][cap] slot of every packed lookup, 0xFFFF = not staged
+    int *pair_ctr;               // [NI]   next run of each (owner, table) pair (reset by the gate)
+};
+
 struct BlsParams {
     int P, T, b, part, S, D, dtype, lanes;
     int NI;                 // number of (owner, table) pairs
@@ -76,6 +93,7 @@ struct BlsParams {
     int *stage_off;              // [S][G+1]
     long long sub_stride;        // NQ + 1 rounded up to a multiple of 4
     long long out_slot_elems;    // P*b*T*D
+    BlsHot hot;
 };
 
 struct bls_plan {
@@ -96,6 +114,8 @@ struct bls_plan {
     int any_stall;                // a delay was injected at some point: ranks may be out of lockstep
     int bags_per_run;             // gather kernel: consecutive sub-bags streamed by one lane group
     int rows_in_flight;           // gather kernel: row loads per batch (4 or 8)
+    long long *h_rows;            // host copy of the table heights
+    int hot_attached;             // a hot-row buffer has been attached
 };
 #define BLS_PROF_MAX 1024
 

@@ -51,6 +51,8 @@ __global__ void __launch_bounds__(32) bls_gate_kernel(BlsParams p, int mode, lon
     const long long BIG = 0x7fffffffffffffffLL;
 
     if (r == 0) d->work_ctr = 0;
+    if (p.hot.enabled)
+        for (int i = r; i < p.NI; i += 32) p.hot.pair_ctr[i] = 0;
     if (r == 0 && (mode == BLS_MODE_STEP || mode == BLS_MODE_ROUTE_ONLY)) {
         int slot = (int)(t_last % p.S);
         d->in_ids[slot] = ids;

@@ -118,11 +118,26 @@ __global__ void __launch_bounds__(256) bls_tw_copy_kernel(BlsParams p)
     const unsigned rows = (unsigned)p.tab[t].rows;
     const int lo = s_lo, hi = max(s_lo, s_hi);
     const int *in = c.ids + off0;
-    for (int l = lo + threadIdx.x; l < hi; l += blockDim.x) {
-        int id = __ldcs(in + l);
-        if ((unsigned)id >= rows) { id = 0; flag(p, BLS_ST_ERANGE); }
-        int pos = cb + l;
-        if (pos < p.cap) c.sendbuf[pos] = id;
+    if (!p.hot.enabled) {
+        for (int l = lo + threadIdx.x; l < hi; l += blockDim.x) {
+            int id = __ldcs(in + l);
+            if ((unsigned)id >= rows) { id = 0; flag(p, BLS_ST_ERANGE); }
+            int pos = cb + l;
+            if (pos < p.cap) c.sendbuf[pos] = id;
+        }
+    } else {
+        // also tell the owner which lookups hit its staged copy of the table's hot rows:
+        // slot = number of hot rows before this one (bitmap + per-word prefix counts)
+        const unsigned *bm = p.hot.bitmap + p.hot.word_base[t], *pf = p.hot.prefix + p.hot.word_base[t];
+        unsigned short *hs = p.hot.hotslot + ((size_t)c.slot * p.P + src) * (size_t)p.cap;
+        for (int l = lo + threadIdx.x; l < hi; l += blockDim.x) {
+            int id = __ldcs(in + l);
+            if ((unsigned)id >= rows) { id = 0; flag(p, BLS_ST_ERANGE); }
+            const unsigned w = __ldg(bm + (id >> 5)), bit = 1u << (id & 31);
+            const unsigned slot = (w & bit) ? __ldg(pf + (id >> 5)) + __popc(w & (bit - 1u)) : 0xFFFFu;
+            int pos = cb + l;
+            if (pos < p.cap) { c.sendbuf[pos] = id; hs[pos] = (unsigned short)slot; }
+        }
     }
 }
 
