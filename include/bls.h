@@ -103,7 +103,8 @@ bls_status_t bls_plan_bytes(const bls_table_t *tables /*host*/, int T, int part,
 
 /* Build a plan inside `workspace` (device, 256-byte aligned, `bytes` long, borrowed
  * until bls_destroy).  Enqueues the initialisation of counters and descriptors on
- * `cuda_stream` (a cudaStream_t; NULL = default stream).  P <= 32, k_max <= 15. */
+ * `cuda_stream` (a cudaStream_t; NULL = default stream).  P <= 32, k_max <= 15, and
+ * T <= 3000 for table-wise placement. */
 bls_status_t bls_plan(const bls_table_t *tables /*host*/, int T, int part, int P, int local_batch,
                       int k_max, int64_t max_ids_per_rank, void *workspace, size_t bytes,
                       void *cuda_stream, bls_plan_t **plan /*host out*/);
@@ -164,8 +165,8 @@ bls_status_t bls_set_wait_limit(bls_plan_t *plan, int64_t ns);
 /* Stage timing with CUDA events on the plan's stream.  While enabled, every
  * bls_step/bls_drain records events around its three stages (up to 1024 calls
  * are kept).  bls_profile_read synchronises the stream, adds up the recorded
- * calls into milliseconds per stage (router kernels, the gather-pool-return
- * kernel, gate + commit kernels), reports how many calls were summed and how
+ * calls into milliseconds per stage (gate + router kernels, the gather-pool-return
+ * kernel including the commit done by its last block, anything after it), reports how many calls were summed and how
  * many kernels they launched, and clears the record.  Any pointer may be NULL. */
 bls_status_t bls_profile(bls_plan_t *plan, int enable);
 bls_status_t bls_profile_read(bls_plan_t *plan, double *ms_route, double *ms_gather, double *ms_ring,

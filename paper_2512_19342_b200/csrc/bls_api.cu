@@ -11,7 +11,7 @@ namespace {
 size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 struct Layout {
-    size_t dev, tab, pair, pair_of, counts, sendbuf, sub_start, out, chunk_base, tile_cnt, stage_ids,
+    size_t dev, tab, pair, pair_of, pair_first, counts, sendbuf, sub_start, out, chunk_base, tile_cnt, stage_ids,
         stage_off, total;
 };
 
@@ -65,6 +65,7 @@ Layout make_layout(const BlsParams &p)
     L.tab = take(sizeof(BlsTableDesc) * p.T);
     L.pair = take(sizeof(BlsPairDesc) * p.NI);
     L.pair_of = take(sizeof(int) * p.T);
+    L.pair_first = take(sizeof(int) * (p.P + 1));
     L.counts = take(sizeof(int) * S * 4 * P * P);
     L.sendbuf = take(sizeof(int) * S * P * (size_t)p.cap);
     L.sub_start = take(sizeof(int) * S * P * (size_t)p.sub_stride);
@@ -129,6 +130,7 @@ bls_status_t bls_plan(const bls_table_t *tables, int T, int part, int P, int loc
     p.tab = (const BlsTableDesc *)(ws + L.tab);
     p.pair = (const BlsPairDesc *)(ws + L.pair);
     p.pair_of_table = (const int *)(ws + L.pair_of);
+    p.pair_first = (const int *)(ws + L.pair_first);
     p.counts = (int *)(ws + L.counts);
     p.sendbuf = (int *)(ws + L.sendbuf);
     p.sub_start = (int *)(ws + L.sub_start);
@@ -163,6 +165,7 @@ bls_status_t bls_plan(const bls_table_t *tables, int T, int part, int P, int loc
     std::vector<BlsTableDesc> tab(T);
     std::vector<BlsPairDesc> pair(p.NI);
     std::vector<int> pair_of(T, 0);
+    std::vector<int> pair_first(P + 1, 0);
     for (int t = 0; t < T; t++) {
         tab[t].weight = tables[t].weight;
         tab[t].rows = tables[t].rows;
@@ -171,6 +174,7 @@ bls_status_t bls_plan(const bls_table_t *tables, int T, int part, int P, int loc
     }
     int n = 0;
     for (int d = 0; d < P; d++) {
+        pair_first[d] = n;
         for (int t = 0; t < T; t++) {
             BlsPairDesc q;
             memset(&q, 0, sizeof(q));
@@ -191,6 +195,7 @@ bls_status_t bls_plan(const bls_table_t *tables, int T, int part, int P, int loc
             pair[n++] = q;
         }
     }
+    pair_first[P] = n;
     BlsDev hd;
     memset(&hd, 0, sizeof(hd));
     for (int r = 0; r < BLS_MAX_RANKS; r++) hd.route_iter[r] = hd.serve_iter[r] = hd.consume_iter[r] = -1;
@@ -201,6 +206,8 @@ bls_status_t bls_plan(const bls_table_t *tables, int T, int part, int P, int loc
               cuda_ok(cudaMemcpyAsync(ws + L.pair, pair.data(), sizeof(BlsPairDesc) * p.NI,
                                       cudaMemcpyHostToDevice, pl->stream)) &&
               cuda_ok(cudaMemcpyAsync(ws + L.pair_of, pair_of.data(), sizeof(int) * T,
+                                      cudaMemcpyHostToDevice, pl->stream)) &&
+              cuda_ok(cudaMemcpyAsync(ws + L.pair_first, pair_first.data(), sizeof(int) * (P + 1),
                                       cudaMemcpyHostToDevice, pl->stream)) &&
               cuda_ok(cudaMemsetAsync(ws + L.counts, 0, sizeof(int) * p.S * 4 * P * P, pl->stream)) &&
               // the vectors above are pageable: make sure the copies have left them
@@ -274,11 +281,9 @@ static void enqueue_wave(bls_plan_t *pl, int mode, long long t_last, long long f
     bls_launch_gate(pl, mode, t_last, floor_, k, ids, off, n_ids);
     bls_launch_route(pl);
     if (ev) cudaEventRecord(ev[1], pl->stream);
-    bls_launch_gather(pl);
-    if (ev) cudaEventRecord(ev[2], pl->stream);
-    bls_launch_commit(pl);
-    if (ev) cudaEventRecord(ev[3], pl->stream);
-    pl->kernels_launched += 3 + bls_route_kernels(pl);
+    bls_launch_gather(pl);                             // its last block commits the wave
+    if (ev) { cudaEventRecord(ev[2], pl->stream); cudaEventRecord(ev[3], pl->stream); }
+    pl->kernels_launched += 2 + bls_route_kernels(pl);
 }
 
 static const float *slot_out(const bls_plan_t *pl, long long iter)
@@ -305,9 +310,8 @@ bls_status_t bls_lookup(bls_plan_t *pl, int64_t iter)
     if (!pl) return BLS_EINVAL;
     if (pl->routed_only != iter) return BLS_ESTATE;
     bls_launch_gate(pl, BLS_MODE_LOOKUP_ONLY, iter, -1, 0, nullptr, nullptr, 0);
-    bls_launch_gather(pl);
-    bls_launch_commit(pl);
-    pl->kernels_launched += 3;
+    bls_launch_gather(pl);                             // its last block commits the wave
+    pl->kernels_launched += 2;
     pl->routed_only = -1;
     pl->t_handed = iter + 1;
     return launch_check();

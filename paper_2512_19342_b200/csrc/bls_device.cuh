@@ -1,0 +1,145 @@
+// Device-side helpers shared by the kernels of libbls (inline: the library is built
+// without relocatable device code).
+#pragma once
+#include "bls_internal.h"
+
+__device__ __forceinline__ unsigned long long globaltimer_ns()
+{
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+
+__device__ __forceinline__ void flag(const BlsParams &p, int bit) { atomicOr(&p.dev->status, bit); }
+
+// What a requester needs to route the iteration the gate assigned to it.
+struct RouteCtx {
+    const int *ids, *off;
+    long long n_ids;
+    int slot;
+    int *sendcounts, *sdispls, *sendbuf, *sub_start;
+};
+
+__device__ __forceinline__ bool route_ctx(const BlsParams &p, int src, RouteCtx &c)
+{
+    long long j = p.dev->route_iter[src];
+    if (j < 0) return false;
+    c.slot = (int)(j % p.S);
+    c.ids = p.dev->in_ids[c.slot];
+    c.off = p.dev->in_off[c.slot];
+    c.n_ids = p.dev->in_n[c.slot];
+    int *cnt = p.counts + (size_t)c.slot * 4 * p.P * p.P;
+    c.sendcounts = cnt + src * p.P;
+    c.sdispls = cnt + p.P * p.P + src * p.P;
+    c.sendbuf = p.sendbuf + ((size_t)c.slot * p.P + src) * (size_t)p.cap;
+    c.sub_start = p.sub_start + ((size_t)c.slot * p.P + src) * (size_t)p.sub_stride;
+    return true;
+}
+
+// Sanitised range of bag g relative to `off0`: 0 <= st <= en <= limit.
+__device__ __forceinline__ bool bag_range(const RouteCtx &c, long long g, long long off0, long long limit,
+                                          int &st, int &en)
+{
+    long long a = (long long)c.off[g] - off0, e = (long long)c.off[g + 1] - off0;
+    bool ok = a >= 0 && a <= e && e <= limit;
+    if (!ok) { a = 0; e = 0; }
+    st = (int)a;
+    en = (int)e;
+    return ok;
+}
+
+// Table-wise router, first half, by one warp for requester `src`: the owner depends
+// on the table only, so the (requester, table) chunks move as a whole.  Chunk
+// lengths come from the offsets alone; an exclusive scan in (owner, table) order
+// gives every chunk its place in the packed send buffer, and the send counts and
+// displacements follow.
+__device__ __forceinline__ void tw_meta_warp(const BlsParams &p, int src, int lane)
+{
+    RouteCtx c;
+    if (!route_ctx(p, src, c)) return;
+    const long long g_rank = (long long)src * p.T * p.b;
+    int *cb = p.chunk_base + (size_t)src * (p.NI + 1);
+    long long run = 0;
+    for (int i0 = 0; i0 < p.NI; i0 += 32) {
+        const int i = i0 + lane;
+        long long n = 0;
+        if (i < p.NI) {
+            const long long g0 = g_rank + (long long)p.pair[i].t * p.b;
+            const long long a = c.off[g0], e = c.off[g0 + p.b];
+            n = e - a;
+            if (a < 0 || n < 0 || e > c.n_ids) { n = 0; flag(p, BLS_ST_EINVAL); }
+        }
+        long long incl = n;
+        for (int o = 1; o < 32; o <<= 1) {
+            const long long y = __shfl_up_sync(0xffffffffu, incl, o);
+            if (lane >= o) incl += y;
+        }
+        if (i < p.NI) cb[i] = (int)min(run + incl - n, (long long)0x7fffffff);
+        run += __shfl_sync(0xffffffffu, incl, 31);
+    }
+    if (lane == 0) {
+        cb[p.NI] = (int)min(run, (long long)0x7fffffff);
+        if (run > p.cap) flag(p, BLS_ST_ENOSPC);
+        c.sub_start[p.NQ] = (int)(run > p.cap ? p.cap : run);
+    }
+    __syncwarp();
+    for (int d = lane; d < p.P; d += 32) {
+        const int lo = cb[p.pair_first[d]], hi = cb[p.pair_first[d + 1]];
+        c.sdispls[d] = lo;
+        c.sendcounts[d] = hi - lo;
+    }
+}
+
+// Publish the progress of the wave that has just run (lane r = rank r) and start the
+// injected delay of every rank that posted.  For every answered iteration also write
+// the receive-side counts and displacements of the request leg (recvcounts =
+// sendcounts transposed, rdispls = exclusive scan over sources).
+__device__ __forceinline__ void commit_lane(const BlsParams &p, int r)
+{
+    BlsDev *d = p.dev;
+    if (r >= p.P) return;
+    const unsigned long long now = globaltimer_ns();
+    long long j = d->route_iter[r];
+    if (j >= 0) {
+        d->posted[r] = j + 1;
+        d->ready_ns[r] = now + d->stall_ns[r];
+        d->route_iter[r] = -1;
+    }
+    j = d->serve_iter[r];
+    if (j >= 0) {
+        int *cnt = p.counts + (size_t)(j % p.S) * 4 * p.P * p.P;
+        const int *sendcounts = cnt;
+        int *recvcounts = cnt + 2 * p.P * p.P, *rdispls = cnt + 3 * p.P * p.P;
+        int run = 0;
+        for (int src = 0; src < p.P; src++) {
+            int c = sendcounts[src * p.P + r];
+            recvcounts[r * p.P + src] = c;
+            rdispls[r * p.P + src] = run;
+            run += c;
+        }
+        d->served[r] = j + 1;
+        d->serve_iter[r] = -1;
+    }
+    j = d->consume_iter[r];
+    if (j >= 0) {
+        d->done[r] = j + 1;
+        d->consume_iter[r] = -1;
+    }
+}
+
+// Called by every thread of every block at the end of the last kernel of a wave:
+// the block that finishes last commits the wave.
+__device__ __forceinline__ void finish_wave(const BlsParams &p)
+{
+    __shared__ int s_last;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        __threadfence();
+        s_last = atomicAdd(&p.dev->done_ctr, 1) == (int)gridDim.x - 1;
+    }
+    __syncthreads();
+    if (s_last && threadIdx.x < 32) {
+        __threadfence();
+        commit_lane(p, threadIdx.x);
+    }
+}

@@ -17,7 +17,7 @@
 #include <cuda_bf16.h>
 #include <cuda_fp16.h>
 #include <type_traits>
-#include "bls_internal.h"
+#include "bls_device.cuh"
 
 // fp32 accumulators as packed pairs: sm_100 adds two fp32 lanes per instruction
 // (round-to-nearest, identical to two scalar adds).
@@ -220,6 +220,7 @@ bls_gather_pool_kernel(BlsParams p, int R, int runs_per_chunk, int n_runs)
         __syncwarp();
         base = __shfl_sync(0xffffffffu, next_base, 0);
     }
+    finish_wave(p);
 }
 
 // Hot-row variant: one persistent block per SM.  Blocks start spread over the
@@ -298,6 +299,7 @@ bls_gather_hot_kernel(BlsParams p, int R, int runs_per_chunk)
             take_runs((i0 + q0 + b) % p.NI, std::false_type{});
         }
     }
+    finish_wave(p);
 }
 
 // Row-wise placement: the IDs of one bag are spread over the owners' regions of the
@@ -394,6 +396,7 @@ bls_gather_rowwise_kernel(BlsParams p, int R, int runs_per_chunk, int n_runs)
         __syncwarp();
         base = __shfl_sync(0xffffffffu, next_base, 0);
     }
+    finish_wave(p);
 }
 
 template <int LANES, int DT, int U>

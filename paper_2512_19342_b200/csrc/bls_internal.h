@@ -35,6 +35,8 @@ struct BlsDev {
     long long max_lag;                            // max over time of newest posted - oldest incomplete
     int status;                                   // OR of BLS_ST_* bits
     int work_ctr;                                 // next run of the gather kernel (reset by the gate)
+    int done_ctr;                                 // blocks of the wave's last kernel that have finished
+    int pad;
 };
 
 struct BlsTableDesc {
@@ -83,6 +85,7 @@ struct BlsParams {
     const BlsTableDesc *tab;     // [T]
     const BlsPairDesc *pair;     // [NI]
     const int *pair_of_table;    // [T] index of table t's (first) pair; row-wise: unused
+    const int *pair_first;       // [P+1] first pair of owner d (pairs are owner-major); [P] = NI
     int *counts;                 // [S][4][P][P]: sendcounts, sdispls, recvcounts, rdispls
     int *sendbuf;                // [S][P][cap]
     int *sub_start;              // [S][P][sub_stride]

@@ -14,14 +14,7 @@
 //     outstanding; the last batch drains everything.
 // A rank under an injected delay takes no action until its delay has passed,
 // unless the bound forces it; then the gate waits (bounded) on the clock.
-#include "bls_internal.h"
-
-__device__ __forceinline__ unsigned long long globaltimer_ns()
-{
-    unsigned long long t;
-    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
-    return t;
-}
+#include "bls_device.cuh"
 
 __device__ __forceinline__ long long warp_min_ll(long long v)
 {
@@ -40,17 +33,18 @@ __device__ __forceinline__ long long warp_max_ll(long long v)
     return v;
 }
 
-// One warp; lane r is logical rank r.
-__global__ void __launch_bounds__(32) bls_gate_kernel(BlsParams p, int mode, long long t_last,
-                                                      long long floor_, int k, const int *ids,
-                                                      const int *off, long long n_ids)
+// Warp 0 decides (lane r is logical rank r).  With table-wise placement the block has
+// one more warp per rank, which then runs the first half of the router for the ranks
+// that were told to post (saves a launch on the critical path of every step).
+__device__ __forceinline__ void gate_warp(const BlsParams &p, int mode, long long t_last, long long floor_, int k,
+                                          const int *ids, const int *off, long long n_ids)
 {
     BlsDev *d = p.dev;
     const int r = threadIdx.x;
     const bool act = r < p.P;
     const long long BIG = 0x7fffffffffffffffLL;
 
-    if (r == 0) d->work_ctr = 0;
+    if (r == 0) { d->work_ctr = 0; d->done_ctr = 0; }
     if (p.hot.enabled)
         for (int i = r; i < p.NI; i += 32) p.hot.pair_ctr[i] = 0;
     if (r == 0 && (mode == BLS_MODE_STEP || mode == BLS_MODE_ROUTE_ONLY)) {
@@ -127,48 +121,28 @@ __global__ void __launch_bounds__(32) bls_gate_kernel(BlsParams p, int mode, lon
     }
 }
 
-// One warp; publishes the progress of the wave that has just run and starts the
-// injected delay of every rank that posted.  For every answered iteration it
-// also writes the receive-side counts and displacements of the request leg
-// (recvcounts = sendcounts transposed, rdispls = exclusive scan over sources).
-__global__ void __launch_bounds__(32) bls_commit_kernel(BlsParams p)
+__global__ void __launch_bounds__(1024) bls_gate_kernel(BlsParams p, int mode, long long t_last,
+                                                        long long floor_, int k, const int *ids,
+                                                        const int *off, long long n_ids)
 {
-    BlsDev *d = p.dev;
-    const int r = threadIdx.x;
-    if (r >= p.P) return;
-    const unsigned long long now = globaltimer_ns();
-    long long j = d->route_iter[r];
-    if (j >= 0) {
-        d->posted[r] = j + 1;
-        d->ready_ns[r] = now + d->stall_ns[r];
-        d->route_iter[r] = -1;
-    }
-    j = d->serve_iter[r];
-    if (j >= 0) {
-        int *cnt = p.counts + (size_t)(j % p.S) * 4 * p.P * p.P;
-        const int *sendcounts = cnt;
-        int *recvcounts = cnt + 2 * p.P * p.P, *rdispls = cnt + 3 * p.P * p.P;
-        int run = 0;
-        for (int src = 0; src < p.P; src++) {
-            int c = sendcounts[src * p.P + r];
-            recvcounts[r * p.P + src] = c;
-            rdispls[r * p.P + src] = run;
-            run += c;
-        }
-        d->served[r] = j + 1;
-        d->serve_iter[r] = -1;
-    }
-    j = d->consume_iter[r];
-    if (j >= 0) {
-        d->done[r] = j + 1;
-        d->consume_iter[r] = -1;
-    }
+    if (threadIdx.x < 32) gate_warp(p, mode, t_last, floor_, k, ids, off, n_ids);
+    if (p.part != BLS_PART_TABLE_RR || mode == BLS_MODE_LOOKUP_ONLY) return;
+    __threadfence_block();
+    __syncthreads();                                   // the wave plan is visible to the other warps
+    const int w = threadIdx.x >> 5;
+    if (w < p.P) tw_meta_warp(p, w, threadIdx.x & 31);
 }
+
+// One warp; publishes the progress of a wave that has no gather kernel at its end
+// (bls_route); otherwise the last block of the gather kernel does this.
+__global__ void __launch_bounds__(32) bls_commit_kernel(BlsParams p) { commit_lane(p, threadIdx.x); }
 
 void bls_launch_gate(const bls_plan_t *pl, int mode, long long t_last, long long forced_floor, int k,
                      const int *ids, const int *off, long long n_ids)
 {
-    bls_gate_kernel<<<1, 32, 0, pl->stream>>>(pl->prm, mode, t_last, forced_floor, k, ids, off, n_ids);
+    // table-wise: one warp per rank for the router's first half (warp 0 is also the gate)
+    const bool meta = pl->prm.part == BLS_PART_TABLE_RR && mode != BLS_MODE_LOOKUP_ONLY;
+    bls_gate_kernel<<<1, meta ? 32 * pl->prm.P : 32, 0, pl->stream>>>(pl->prm, mode, t_last, forced_floor, k, ids, off, n_ids);
 }
 
 void bls_launch_commit(const bls_plan_t *pl)

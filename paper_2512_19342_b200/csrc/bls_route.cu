@@ -12,82 +12,12 @@
 // Table-wise placement: the owner depends on the table only, so a requester's
 // (table) chunks move as a whole; counts follow from the offsets alone.
 // Row-wise placement: a real multisplit, done per tile of 128 bags of one table.
-#include "bls_internal.h"
-
-__device__ __forceinline__ void flag(const BlsParams &p, int bit) { atomicOr(&p.dev->status, bit); }
-
-struct RouteCtx {
-    const int *ids, *off;
-    long long n_ids;
-    int slot;
-    int *sendcounts, *sdispls, *sendbuf, *sub_start;
-};
-
-__device__ __forceinline__ bool route_ctx(const BlsParams &p, int src, RouteCtx &c)
-{
-    long long j = p.dev->route_iter[src];
-    if (j < 0) return false;
-    c.slot = (int)(j % p.S);
-    c.ids = p.dev->in_ids[c.slot];
-    c.off = p.dev->in_off[c.slot];
-    c.n_ids = p.dev->in_n[c.slot];
-    int *cnt = p.counts + (size_t)c.slot * 4 * p.P * p.P;
-    c.sendcounts = cnt + src * p.P;
-    c.sdispls = cnt + p.P * p.P + src * p.P;
-    c.sendbuf = p.sendbuf + ((size_t)c.slot * p.P + src) * (size_t)p.cap;
-    c.sub_start = p.sub_start + ((size_t)c.slot * p.P + src) * (size_t)p.sub_stride;
-    return true;
-}
-
-// Sanitised range of bag g relative to rank base `off0`: 0 <= st <= en <= limit.
-__device__ __forceinline__ bool bag_range(const RouteCtx &c, long long g, long long off0, long long limit,
-                                          int &st, int &en)
-{
-    long long a = (long long)c.off[g] - off0, e = (long long)c.off[g + 1] - off0;
-    bool ok = a >= 0 && a <= e && e <= limit;
-    if (!ok) { a = 0; e = 0; }
-    st = (int)a;
-    en = (int)e;
-    return ok;
-}
+#include "bls_device.cuh"
 
 // ------------------------------------------------------------------ table-wise
-
-// One block per requester: chunk lengths from the offsets, exclusive scan in
-// (owner, table) order, send counts and displacements.
-__global__ void __launch_bounds__(128) bls_tw_meta_kernel(BlsParams p)
-{
-    extern __shared__ int len[];                 // [NI]
-    const int src = blockIdx.x;
-    RouteCtx c;
-    if (!route_ctx(p, src, c)) return;
-    const long long g_rank = (long long)src * p.T * p.b;
-    const long long off_rank = c.off[g_rank];
-    for (int i = threadIdx.x; i < p.NI; i += blockDim.x) {
-        long long g0 = g_rank + (long long)p.pair[i].t * p.b;
-        long long a = c.off[g0], e = c.off[g0 + p.b];
-        long long n = e - a;
-        if (a < 0 || n < 0 || e > c.n_ids) { n = 0; flag(p, BLS_ST_EINVAL); }
-        len[i] = (int)n;
-    }
-    __syncthreads();
-    if (threadIdx.x == 0) {
-        int *cb = p.chunk_base + (size_t)src * (p.NI + 1);
-        long long run = 0;
-        int i = 0;
-        for (int d = 0; d < p.P; d++) {
-            c.sdispls[d] = (int)run;
-            long long before = run;
-            while (i < p.NI && p.pair[i].dst == d) { cb[i] = (int)run; run += len[i]; i++; }
-            c.sendcounts[d] = (int)(run - before);
-        }
-        cb[p.NI] = (int)run;
-        if (run > p.cap) flag(p, BLS_ST_ENOSPC);
-        c.sub_start[p.NQ] = (int)(run > p.cap ? p.cap : run);
-        (void)off_rank;
-    }
-}
-
+// First half (chunk lengths, scan, counts, displacements): tw_meta_warp, run by the
+// gate kernel.  Second half, here: move every ID to its place and write the sub-bag
+// starts.
 // grid (NT, P): tile = 128 bags of one (requester, table) chunk.  Copies the
 // chunk's IDs to their place in the send buffer (coalesced) and writes the
 // sub-bag starts.
@@ -119,11 +49,22 @@ __global__ void __launch_bounds__(256) bls_tw_copy_kernel(BlsParams p)
     const int lo = s_lo, hi = max(s_lo, s_hi);
     const int *in = c.ids + off0;
     if (!p.hot.enabled) {
-        for (int l = lo + threadIdx.x; l < hi; l += blockDim.x) {
-            int id = __ldcs(in + l);
-            if ((unsigned)id >= rows) { id = 0; flag(p, BLS_ST_ERANGE); }
-            int pos = cb + l;
-            if (pos < p.cap) c.sendbuf[pos] = id;
+        for (int l0 = lo + threadIdx.x; l0 < hi; l0 += 4 * blockDim.x) {
+            int id[4];
+            #pragma unroll
+            for (int q = 0; q < 4; q++) {
+                const int l = l0 + q * blockDim.x;
+                id[q] = l < hi ? __ldcs(in + l) : 0;
+            }
+            #pragma unroll
+            for (int q = 0; q < 4; q++) {
+                const int l = l0 + q * blockDim.x;
+                if (l >= hi) continue;
+                int v = id[q];
+                if ((unsigned)v >= rows) { v = 0; flag(p, BLS_ST_ERANGE); }
+                const int pos = cb + l;
+                if (pos < p.cap) c.sendbuf[pos] = v;
+            }
         }
     } else {
         // also tell the owner which lookups hit its staged copy of the table's hot rows:
@@ -285,14 +226,13 @@ __global__ void __launch_bounds__(BLS_ROUTE_TB) bls_rw_scatter_kernel(BlsParams 
     }
 }
 
-int bls_route_kernels(const bls_plan_t *pl) { return pl->prm.part == BLS_PART_TABLE_RR ? 2 : 3; }
+int bls_route_kernels(const bls_plan_t *pl) { return pl->prm.part == BLS_PART_TABLE_RR ? 1 : 3; }
 
 void bls_launch_route(const bls_plan_t *pl)
 {
     const BlsParams &p = pl->prm;
     dim3 grid(p.NT, p.P);
     if (p.part == BLS_PART_TABLE_RR) {
-        bls_tw_meta_kernel<<<p.P, 128, p.NI * sizeof(int), pl->stream>>>(p);
         bls_tw_copy_kernel<<<grid, 256, 0, pl->stream>>>(p);
     } else {
         bls_rw_count_kernel<<<grid, BLS_ROUTE_TB, 0, pl->stream>>>(p);
