@@ -170,7 +170,7 @@ bls_status_t bls_plan(const bls_table_t *tables, int T, int part, int P, int loc
         tab[t].weight = tables[t].weight;
         tab[t].rows = tables[t].rows;
         tab[t].blk = part == BLS_PART_ROW_BLOCK ? (int)((tables[t].rows + P - 1) / P) : 0;
-        tab[t].pad = 0;
+        tab[t].magic = tab[t].blk <= 1 ? 0xFFFFFFFFu : (unsigned)((1ull << 32) / (unsigned long long)tab[t].blk);
     }
     int n = 0;
     for (int d = 0; d < P; d++) {

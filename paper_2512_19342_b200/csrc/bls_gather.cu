@@ -403,9 +403,14 @@ template <int LANES, int DT, int U>
 static void launch_gather(const bls_plan_t *pl)
 {
     const BlsParams &p = pl->prm;
-    const int R = pl->bags_per_run;
-    const int rpc = (p.b + R - 1) / R;
     const bool rowwise = p.part == BLS_PART_ROW_BLOCK;
+    // Runs are as long as the plan asks for, but short enough that every resident lane
+    // group gets at least two: small workloads are latency-bound and need the parallelism.
+    const long long bags = (long long)(rowwise ? p.T : p.NI) * p.P * p.b;
+    const long long resident_groups = (long long)pl->sm_count * 24 * (32 / LANES);
+    long long fit = bags / (2 * resident_groups);
+    const int R = (int)(fit < 1 ? 1 : (fit < pl->bags_per_run ? fit : pl->bags_per_run));
+    const int rpc = (p.b + R - 1) / R;
     // table-wise: runs of sub-bags of one (owner, table, requester); row-wise: runs of bags of one (table, requester)
     const long long n_runs = (long long)(rowwise ? p.T : p.NI) * p.P * rpc;
     // more blocks than fit at once (late ones find the counter exhausted), fewer for small workloads

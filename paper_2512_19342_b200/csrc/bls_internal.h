@@ -43,7 +43,7 @@ struct BlsTableDesc {
     const void *weight;
     long long rows;
     int blk;            // ceil(rows / P) for row-block placement, else 0
-    int pad;
+    unsigned magic;     // floor(2^32 / blk) (2^32 - 1 for blk = 1): division by blk as a multiply
 };
 
 // A (owner, table) pair in owner-major order.  Table-wise: one pair per table.
