@@ -342,55 +342,135 @@ bls_gather_rowwise_kernel(BlsParams p, int R, int runs_per_chunk, int n_runs)
                             ((size_t)t * p.b + s0) * p.P;
             float *o = p.out + (size_t)slot * p.out_slot_elems +
                        (((size_t)src * p.b + s0) * p.T + t) * p.D + lane * Acc<DT>::N;
-            for (int bag = 0; bag < nb; bag++, ss += p.P, o += (size_t)p.T * p.D) {
-                Acc<DT> acc;
-                acc.zero();
-                for (int c0 = 0; c0 < p.P; c0 += LANES) {      // owners c0 .. c0+LANES-1, one per lane
-                    const int d = c0 + lane;
-                    int st = 0, en = 0;
-                    if (d < p.P) {
-                        st = min(max(ss[d], 0), p.cap);
-                        en = min(max(ss[p.P + d], st), p.cap);
-                    }
-                    const int n = en - st;
-                    int incl = n;                               // inclusive scan over the group's lanes
+            if (p.P <= LANES) {
+                // All owners fit in one lane group (lane d = owner d).  Three bags are in
+                // flight: while the rows of bag k are loaded and added, the IDs of bag k+1
+                // are already on their way and the bounds of bags k+2, k+3 are being fetched,
+                // so only the row loads are ever waited for.
+                const int d = lane;
+                const bool own_lane = d < p.P;
+                auto bound = [&](int k) { return own_lane ? min(max(ss[(size_t)k * p.P + d], 0), p.cap) : 0; };
+                struct Pre { int idv, own, total, st, excl; };
+                auto prepare = [&](int st, int en_raw) {        // scan the owners' counts, fetch this lane's ID
+                    Pre q;
+                    const int n = max(en_raw - st, 0);
+                    int incl = n;
                     #pragma unroll
                     for (int w = 1; w < LANES; w <<= 1) {
                         const int y = __shfl_up_sync(gmask, incl, w, LANES);
                         if (lane >= w) incl += y;
                     }
-                    const int excl = incl - n;
-                    const int total = __shfl_sync(gmask, incl, LANES - 1, LANES);
-                    for (int r0 = 0; r0 < total; r0 += LANES) {
-                        const int r = r0 + lane;                // this lane fetches the ID of row r
-                        int own = 0;                            // last lane whose first row is <= r
+                    q.st = st;
+                    q.excl = incl - n;
+                    q.total = __shfl_sync(gmask, incl, LANES - 1, LANES);
+                    int own = 0;                                // last lane whose first row is <= lane
+                    #pragma unroll
+                    for (int step = LANES / 2; step >= 1; step >>= 1) {
+                        const int ex = __shfl_sync(gmask, q.excl, own + step, LANES);
+                        if (ex <= lane) own += step;
+                    }
+                    const int pos = __shfl_sync(gmask, st, own, LANES) + lane - __shfl_sync(gmask, q.excl, own, LANES);
+                    q.own = own;
+                    q.idv = lane < q.total ? __ldcs(sb + min(pos, p.cap - 1)) : 0;
+                    return q;
+                };
+                int r0v = bound(0), r1v = bound(1);
+                int r2v = nb >= 2 ? bound(2) : 0;
+                Pre cur = prepare(r0v, r1v);
+                int st_n = r1v, en_n = r2v;                     // bounds of bag 1
+                for (int bag = 0; bag < nb; bag++, o += (size_t)p.T * p.D) {
+                    const int r3v = bag + 3 <= nb ? bound(bag + 3) : 0;            // bounds two bags ahead
+                    Pre nxt = cur;
+                    if (bag + 1 < nb) nxt = prepare(st_n, en_n);                   // IDs one bag ahead
+                    Acc<DT> acc;
+                    acc.zero();
+                    const unsigned grow = min((unsigned)cur.own * (unsigned)tb.blk + (unsigned)cur.idv, rows_m1);
+                    const int m = min(LANES, cur.total);
+                    #pragma unroll 1
+                    for (int u0 = 0; u0 < m; u0 += U) {
+                        uint4 v[U];
+                        #pragma unroll
+                        for (int u = 0; u < U; u++) {
+                            const unsigned row = __shfl_sync(gmask, grow, u0 + u, LANES);
+                            v[u] = (u0 + u < m) ? __ldg(rowbase + (size_t)row * LANES) : make_uint4(0u, 0u, 0u, 0u);
+                        }
+                        #pragma unroll
+                        for (int u = 0; u < U; u++)
+                            if (u0 + u < m) acc.add(v[u]);
+                    }
+                    for (int r0 = LANES; r0 < cur.total; r0 += LANES) {           // rare: more rows than lanes
+                        const int r = r0 + lane;
+                        int own = 0;
                         #pragma unroll
                         for (int step = LANES / 2; step >= 1; step >>= 1) {
-                            const int ex = __shfl_sync(gmask, excl, own + step, LANES);
+                            const int ex = __shfl_sync(gmask, cur.excl, own + step, LANES);
                             if (ex <= r) own += step;
                         }
-                        const int pos = __shfl_sync(gmask, st, own, LANES) + r - __shfl_sync(gmask, excl, own, LANES);
-                        unsigned grow = 0;
-                        if (r < total) {
-                            const unsigned id = (unsigned)__ldcs(sb + pos);
-                            grow = min((unsigned)(c0 + own) * (unsigned)tb.blk + id, rows_m1);
-                        }
-                        const int m = min(LANES, total - r0);
-                        #pragma unroll 1
-                        for (int u0 = 0; u0 < m; u0 += U) {
-                            uint4 v[U];
-                            #pragma unroll
-                            for (int u = 0; u < U; u++) {
-                                const unsigned row = __shfl_sync(gmask, grow, u0 + u, LANES);
-                                v[u] = (u0 + u < m) ? __ldg(rowbase + (size_t)row * LANES) : make_uint4(0u, 0u, 0u, 0u);
-                            }
-                            #pragma unroll
-                            for (int u = 0; u < U; u++)
-                                if (u0 + u < m) acc.add(v[u]);
+                        const int pos = __shfl_sync(gmask, cur.st, own, LANES) + r - __shfl_sync(gmask, cur.excl, own, LANES);
+                        unsigned g2 = 0;
+                        if (r < cur.total) g2 = min((unsigned)own * (unsigned)tb.blk + (unsigned)__ldcs(sb + min(pos, p.cap - 1)), rows_m1);
+                        const int m2 = min(LANES, cur.total - r0);
+                        for (int u = 0; u < m2; u++) {
+                            const unsigned row = __shfl_sync(gmask, g2, u, LANES);
+                            acc.add(__ldg(rowbase + (size_t)row * LANES));
                         }
                     }
+                    flush<DT>(o, acc);
+                    cur = nxt;
+                    st_n = en_n;
+                    en_n = r3v;
                 }
-                flush<DT>(o, acc);
+            } else {
+                for (int bag = 0; bag < nb; bag++, ss += p.P, o += (size_t)p.T * p.D) {
+                    Acc<DT> acc;
+                    acc.zero();
+                    for (int c0 = 0; c0 < p.P; c0 += LANES) {      // owners c0 .. c0+LANES-1, one per lane
+                        const int d = c0 + lane;
+                        int st = 0, en = 0;
+                        if (d < p.P) {
+                            st = min(max(ss[d], 0), p.cap);
+                            en = min(max(ss[p.P + d], st), p.cap);
+                        }
+                        const int n = en - st;
+                        int incl = n;                               // inclusive scan over the group's lanes
+                        #pragma unroll
+                        for (int w = 1; w < LANES; w <<= 1) {
+                            const int y = __shfl_up_sync(gmask, incl, w, LANES);
+                            if (lane >= w) incl += y;
+                        }
+                        const int excl = incl - n;
+                        const int total = __shfl_sync(gmask, incl, LANES - 1, LANES);
+                        for (int r0 = 0; r0 < total; r0 += LANES) {
+                            const int r = r0 + lane;                // this lane fetches the ID of row r
+                            int own = 0;                            // last lane whose first row is <= r
+                            #pragma unroll
+                            for (int step = LANES / 2; step >= 1; step >>= 1) {
+                                const int ex = __shfl_sync(gmask, excl, own + step, LANES);
+                                if (ex <= r) own += step;
+                            }
+                            const int pos = __shfl_sync(gmask, st, own, LANES) + r - __shfl_sync(gmask, excl, own, LANES);
+                            unsigned grow = 0;
+                            if (r < total) {
+                                const unsigned id = (unsigned)__ldcs(sb + pos);
+                                grow = min((unsigned)(c0 + own) * (unsigned)tb.blk + id, rows_m1);
+                            }
+                            const int m = min(LANES, total - r0);
+                            #pragma unroll 1
+                            for (int u0 = 0; u0 < m; u0 += U) {
+                                uint4 v[U];
+                                #pragma unroll
+                                for (int u = 0; u < U; u++) {
+                                    const unsigned row = __shfl_sync(gmask, grow, u0 + u, LANES);
+                                    v[u] = (u0 + u < m) ? __ldg(rowbase + (size_t)row * LANES) : make_uint4(0u, 0u, 0u, 0u);
+                                }
+                                #pragma unroll
+                                for (int u = 0; u < U; u++)
+                                    if (u0 + u < m) acc.add(v[u]);
+                            }
+                        }
+                    }
+                    flush<DT>(o, acc);
+                }
             }
         }
         __syncwarp();
