@@ -48,6 +48,8 @@ def parse_args():
     ap.add_argument("--tune", default="", help="bags_per_run,rows_in_flight for the gather kernel (0 = default)")
     ap.add_argument("--hot", type=int, default=-1,
                     help="hot rows per table staged in shared memory (0 = off, -1 = the workload's default)")
+    ap.add_argument("--delay-us", type=float, default=0.0,
+                    help="also time the loop with a uniform random delay in [0, 2*D] us per rank and iteration")
     ap.add_argument("--ks", default="", help="comma-separated bounds to time instead of the workload's own")
     return ap.parse_args()
 
@@ -390,6 +392,20 @@ def run_mine(args):
         e2e = {"value": tot_e / (ms_e * 1e-3), "unit": "lookups/s",
                "h2d_bytes_per_step": int(np.mean([i.nbytes + o.nbytes for i, o in inputs])),
                "d2h_bytes_per_step": int(h_out.numel() * 4), "steps": n_e2e, "k": k_head}
+    delay_sweep = None
+    if args.delay_us > 0:
+        # the paper's random-delay setting: bound 0 pays the largest delay every iteration, k > 0 hides part of it
+        delay_sweep = {}
+        for r in range(w.P):
+            bls.bls_set_random_stall(plan, r, int(2 * args.delay_us * 1000), 2024)
+        bls.bls_set_waves_per_step(plan, w.P + 1)
+        for k in ks:
+            ms, _ = aggregate(timed(k, args.steps), units, world, dev)
+            delay_sweep[str(k)] = {"ms_per_step": ms / args.steps}
+        for r in range(w.P):
+            bls.bls_set_random_stall(plan, r, 0, 2024)
+        delay_sweep["mean_delay_us"] = args.delay_us
+        delay_sweep["expected_k0_extra_us"] = 2 * args.delay_us * w.P / (w.P + 1)
     clocks = sampler.stop() if sampler else None
     st, lag = bls.bls_status(plan)
     if st != bls.BLS_OK:
@@ -425,7 +441,7 @@ def run_mine(args):
                      "bytes_per_launch": gather_bytes, "ms_per_launch": ms_gather, "peak_source": peak_src},
         "stage_ms_per_step": {"route": prof["ms_route"] / max(1, prof["calls"]), "gather_pool_return": ms_gather,
                               "ring": prof["ms_ring"] / max(1, prof["calls"])},
-        "clocks": clocks, "e2e": e2e, "gpu_launches": launches,
+        "clocks": clocks, "e2e": e2e, "gpu_launches": launches, "delay_sweep": delay_sweep,
     }
     if not args.no_cpu_baseline and world == 1:
         result["cpu_baseline"] = cpu_baseline(w, inputs)

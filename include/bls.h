@@ -159,6 +159,15 @@ bls_status_t bls_status(bls_plan_t *plan, int64_t *max_lag /*host out*/);
 /* Injected delay of rank `rank` before each of its iterations (Section V-E,
  * setting 2: a delay models a slowdown of any nature), in nanoseconds. */
 bls_status_t bls_set_stall(bls_plan_t *plan, int rank, int64_t ns);
+/* The paper's random-delay setting: in addition to the fixed delay, rank `rank` is
+ * delayed before each of its iterations by a time drawn uniformly from [0, max_ns]
+ * (a counter-based draw from `seed`, the rank and the iteration number, so a run
+ * can be repeated).  The seed is shared by all ranks of the plan. */
+bls_status_t bls_set_random_stall(bls_plan_t *plan, int rank, int64_t max_ns, uint64_t seed);
+/* While delays are injected, one bls_step runs up to `waves` waves of kernels (default 4,
+ * at most P+1): all but the last wait only for the earliest rank that can act, which lets
+ * ranks act at different moments and catch up; the last one enforces the bound. */
+bls_status_t bls_set_waves_per_step(bls_plan_t *plan, int waves);
 /* Upper limit of any single device-side wait (default 2 s). */
 bls_status_t bls_set_wait_limit(bls_plan_t *plan, int64_t ns);
 

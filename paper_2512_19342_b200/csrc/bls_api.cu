@@ -152,6 +152,7 @@ bls_status_t bls_plan(const bls_table_t *tables, int T, int part, int P, int loc
         int R = (int)(320.0 / (avg < 0.5 ? 0.5 : avg) + 0.5);
         pl->bags_per_run = R < 4 ? 4 : (R > 64 ? 64 : R);
         pl->rows_in_flight = 4;
+        pl->max_waves = 4;
     }
     int devid = 0;
     if (!cuda_ok(cudaGetDevice(&devid)) ||
@@ -266,7 +267,7 @@ static bls_status_t launch_check()
 
 // One wave: gate -> router -> gather/pool/return -> commit, with optional stage events.
 static void enqueue_wave(bls_plan_t *pl, int mode, long long t_last, long long floor_, int k,
-                         const int *ids, const int *off, long long n_ids)
+                         const int *ids, const int *off, long long n_ids, int opportunistic = 0)
 {
     cudaEvent_t *ev = nullptr;
     if (pl->prof_on && pl->prof_n < BLS_PROF_MAX) {
@@ -278,7 +279,7 @@ static void enqueue_wave(bls_plan_t *pl, int mode, long long t_last, long long f
         if (pl->prof_ev) ev = pl->prof_ev + (size_t)pl->prof_n++ * 4;
     }
     if (ev) cudaEventRecord(ev[0], pl->stream);
-    bls_launch_gate(pl, mode, t_last, floor_, k, ids, off, n_ids);
+    bls_launch_gate(pl, mode, t_last, floor_, k, ids, off, n_ids, opportunistic);
     bls_launch_route(pl);
     if (ev) cudaEventRecord(ev[1], pl->stream);
     bls_launch_gather(pl);                             // its last block commits the wave
@@ -296,7 +297,7 @@ bls_status_t bls_route(bls_plan_t *pl, int64_t iter, const int32_t *ids, const i
 {
     if (!pl || !offsets || (!ids && n_ids > 0) || n_ids < 0) return BLS_EINVAL;
     if (iter != pl->t_next || pl->t_handed != pl->t_next || pl->routed_only >= 0) return BLS_ESTATE;
-    bls_launch_gate(pl, BLS_MODE_ROUTE_ONLY, iter, -1, 0, ids, offsets, n_ids);
+    bls_launch_gate(pl, BLS_MODE_ROUTE_ONLY, iter, -1, 0, ids, offsets, n_ids, 0);
     bls_launch_route(pl);
     bls_launch_commit(pl);
     pl->kernels_launched += 2 + bls_route_kernels(pl);
@@ -309,7 +310,7 @@ bls_status_t bls_lookup(bls_plan_t *pl, int64_t iter)
 {
     if (!pl) return BLS_EINVAL;
     if (pl->routed_only != iter) return BLS_ESTATE;
-    bls_launch_gate(pl, BLS_MODE_LOOKUP_ONLY, iter, -1, 0, nullptr, nullptr, 0);
+    bls_launch_gate(pl, BLS_MODE_LOOKUP_ONLY, iter, -1, 0, nullptr, nullptr, 0, 0);
     bls_launch_gather(pl);                             // its last block commits the wave
     pl->kernels_launched += 2;
     pl->routed_only = -1;
@@ -325,7 +326,13 @@ bls_status_t bls_step(bls_plan_t *pl, int k, const int32_t *ids, const int32_t *
     if (pl->k_cur >= 0 && pl->k_cur != k && pl->t_handed != pl->t_next) return BLS_ESTATE;
     pl->k_cur = k;
     const long long t = pl->t_next++;
-    enqueue_wave(pl, BLS_MODE_STEP, t, t - k, k, ids, offsets, n_ids);
+    // With injected delays the ranks act at different moments: a few opportunistic waves
+    // (while the iteration to hand back is incomplete they wait for the earliest rank that can act) let them drift apart and catch
+    // up, the last wave enforces the bound.  Without delays one wave does everything.
+    const int waves = pl->any_stall ? (pl->max_waves < pl->prm.P + 1 ? pl->max_waves : pl->prm.P + 1) : 1;
+    for (int v = 0; v + 1 < waves; v++)
+        enqueue_wave(pl, BLS_MODE_STEP, t, t - k, k, ids, v == 0 ? offsets : nullptr, n_ids, 1);
+    enqueue_wave(pl, BLS_MODE_STEP, t, t - k, k, ids, waves == 1 ? offsets : nullptr, n_ids);
     if (t - k >= 0) {
         *out = slot_out(pl, t - k);
         *out_iter = t - k;
@@ -459,6 +466,25 @@ bls_status_t bls_set_stall(bls_plan_t *pl, int rank, int64_t ns)
                    cudaStreamSynchronize(pl->stream) == cudaSuccess
                ? BLS_OK
                : BLS_ECUDA;
+}
+
+bls_status_t bls_set_random_stall(bls_plan_t *pl, int rank, int64_t max_ns, uint64_t seed)
+{
+    if (!pl || rank < 0 || rank >= pl->prm.P || max_ns < 0) return BLS_EINVAL;
+    unsigned long long v = (unsigned long long)max_ns, sd = seed;
+    if (max_ns > 0) pl->any_stall = 1;
+    return cudaMemcpyAsync(&pl->prm.dev->stall_rand_ns[rank], &v, sizeof(v), cudaMemcpyHostToDevice, pl->stream) == cudaSuccess &&
+                   cudaMemcpyAsync(&pl->prm.dev->stall_seed, &sd, sizeof(sd), cudaMemcpyHostToDevice, pl->stream) == cudaSuccess &&
+                   cudaStreamSynchronize(pl->stream) == cudaSuccess
+               ? BLS_OK
+               : BLS_ECUDA;
+}
+
+bls_status_t bls_set_waves_per_step(bls_plan_t *pl, int waves)
+{
+    if (!pl || waves < 1 || waves > 64) return BLS_EINVAL;
+    pl->max_waves = waves;
+    return BLS_OK;
 }
 
 bls_status_t bls_set_tuning(bls_plan_t *pl, int bags_per_run, int rows_in_flight)

@@ -102,7 +102,17 @@ __device__ __forceinline__ void commit_lane(const BlsParams &p, int r)
     long long j = d->route_iter[r];
     if (j >= 0) {
         d->posted[r] = j + 1;
-        d->ready_ns[r] = now + d->stall_ns[r];
+        unsigned long long stall = d->stall_ns[r];
+        const unsigned long long span = d->stall_rand_ns[r];
+        if (span) {
+            // uniform in [0, span]: SplitMix64 output for (seed, rank, iteration), a counter-based draw
+            unsigned long long z = d->stall_seed + (((unsigned long long)r << 40) + (unsigned long long)j + 1ull) * 0x9E3779B97F4A7C15ull;
+            z = (z ^ (z >> 30)) * 0xBF58476D1CE4E5B9ull;
+            z = (z ^ (z >> 27)) * 0x94D049BB133111EBull;
+            z ^= z >> 31;
+            stall += z % (span + 1ull);
+        }
+        d->ready_ns[r] = now + stall;
         d->route_iter[r] = -1;
     }
     j = d->serve_iter[r];

@@ -23,6 +23,8 @@ struct BlsDev {
     long long done[BLS_MAX_RANKS];
     unsigned long long ready_ns[BLS_MAX_RANKS];   // rank may act again at this globaltimer value
     unsigned long long stall_ns[BLS_MAX_RANKS];   // injected delay before each iteration
+    unsigned long long stall_rand_ns[BLS_MAX_RANKS];  // plus a uniform random part in [0, this]
+    unsigned long long stall_seed;                // seed of the counter-based generator for the random part
     // plan of the current wave: iteration each rank routes / serves / completes, or -1
     long long route_iter[BLS_MAX_RANKS];
     long long serve_iter[BLS_MAX_RANKS];
@@ -118,13 +120,14 @@ struct bls_plan {
     int bags_per_run;             // gather kernel: consecutive sub-bags streamed by one lane group
     int rows_in_flight;           // gather kernel: row loads per batch (4 or 8)
     long long *h_rows;            // host copy of the table heights
+    int max_waves;                // with injected delays: waves per step (the last one enforces the bound)
     int hot_attached;             // a hot-row buffer has been attached
 };
 #define BLS_PROF_MAX 1024
 
 // kernel launchers (defined in the .cu files)
 void bls_launch_gate(const bls_plan_t *pl, int mode, long long t_last, long long forced_floor, int k,
-                     const int *ids, const int *off, long long n_ids);
+                     const int *ids, const int *off, long long n_ids, int opportunistic);
 void bls_launch_commit(const bls_plan_t *pl);
 void bls_launch_route(const bls_plan_t *pl);
 void bls_launch_gather(const bls_plan_t *pl);

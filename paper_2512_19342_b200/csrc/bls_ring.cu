@@ -37,7 +37,7 @@ __device__ __forceinline__ long long warp_max_ll(long long v)
 // one more warp per rank, which then runs the first half of the router for the ranks
 // that were told to post (saves a launch on the critical path of every step).
 __device__ __forceinline__ void gate_warp(const BlsParams &p, int mode, long long t_last, long long floor_, int k,
-                                          const int *ids, const int *off, long long n_ids)
+                                          const int *ids, const int *off, long long n_ids, int opportunistic)
 {
     BlsDev *d = p.dev;
     const int r = threadIdx.x;
@@ -47,7 +47,7 @@ __device__ __forceinline__ void gate_warp(const BlsParams &p, int mode, long lon
     if (r == 0) { d->work_ctr = 0; d->done_ctr = 0; }
     if (p.hot.enabled)
         for (int i = r; i < p.NI; i += 32) p.hot.pair_ctr[i] = 0;
-    if (r == 0 && (mode == BLS_MODE_STEP || mode == BLS_MODE_ROUTE_ONLY)) {
+    if (r == 0 && off != nullptr && (mode == BLS_MODE_STEP || mode == BLS_MODE_ROUTE_ONLY)) {
         int slot = (int)(t_last % p.S);
         d->in_ids[slot] = ids;
         d->in_off[slot] = off;
@@ -61,16 +61,32 @@ __device__ __forceinline__ void gate_warp(const BlsParams &p, int mode, long lon
     unsigned long long ready_at = act ? d->ready_ns[r] : 0ull;
     const bool sync_mode = (mode == BLS_MODE_ROUTE_ONLY || mode == BLS_MODE_LOOKUP_ONLY);
 
-    // Ranks the bound forces to act in this wave: anything still at or below the floor.
-    bool forced = act && (sync_mode || (floor_ >= 0 && (posted <= floor_ || served <= floor_ || done <= floor_)));
-
-    // Bounded wait on the clock for the forced ranks' injected delays.
+    // Ranks the bound forces to act: anything still at or below the floor.  Only the last
+    // wave of a step forces them (and waits, bounded, for their injected delays).  An earlier
+    // wave waits only while the step's obligation - everything up to the floor complete - is
+    // unmet, and then only for the earliest rank that could act, so that faster ranks keep
+    // running ahead while a slow one is awaited; once the obligation is met it never waits.
+    const bool at_floor = act && floor_ >= 0 && (posted <= floor_ || served <= floor_ || done <= floor_);
+    const bool forced = act && (sync_mode || (!opportunistic && at_floor));
     unsigned long long need = forced ? ready_at : 0ull;
     for (int o = 16; o > 0; o >>= 1) {
         unsigned long long w = __shfl_xor_sync(0xffffffffu, need, o);
         need = w > need ? w : need;
     }
     unsigned long long now = globaltimer_ns();
+    if (opportunistic) {
+        need = 0ull;
+        if (__any_sync(0xffffffffu, at_floor)) {
+            const long long mp = warp_min_ll(posted), ms = warp_min_ll(served), md = warp_min_ll(done);
+            const bool could = act && ((posted <= t_last && md >= posted - k) || served < mp || done < ms);
+            unsigned long long first = could ? ready_at : ~0ull;
+            for (int o = 16; o > 0; o >>= 1) {
+                unsigned long long w = __shfl_xor_sync(0xffffffffu, first, o);
+                first = w < first ? w : first;
+            }
+            need = first == ~0ull ? 0ull : first;
+        }
+    }
     if (!sync_mode && need > now) {
         const unsigned long long give_up = now + d->wait_limit_ns;
         while (now < need && now < give_up) {
@@ -115,7 +131,7 @@ __device__ __forceinline__ void gate_warp(const BlsParams &p, int mode, long lon
         long long lag = max_posted2 - 1 - min_done;
         if (lag > d->max_lag) d->max_lag = lag;
         // the wave must satisfy the bound: everything up to the floor completes
-        if (!sync_mode && floor_ >= 0 && min_done2 <= floor_) atomicOr(&d->status, BLS_ST_ESTATE);
+        if (!sync_mode && !opportunistic && floor_ >= 0 && min_done2 <= floor_) atomicOr(&d->status, BLS_ST_ESTATE);
         if (mode == BLS_MODE_ROUTE_ONLY && min_posted2 <= t_last) atomicOr(&d->status, BLS_ST_ESTATE);
         if (mode == BLS_MODE_LOOKUP_ONLY && min_done2 <= t_last) atomicOr(&d->status, BLS_ST_ESTATE);
     }
@@ -123,9 +139,9 @@ __device__ __forceinline__ void gate_warp(const BlsParams &p, int mode, long lon
 
 __global__ void __launch_bounds__(1024) bls_gate_kernel(BlsParams p, int mode, long long t_last,
                                                         long long floor_, int k, const int *ids,
-                                                        const int *off, long long n_ids)
+                                                        const int *off, long long n_ids, int opportunistic)
 {
-    if (threadIdx.x < 32) gate_warp(p, mode, t_last, floor_, k, ids, off, n_ids);
+    if (threadIdx.x < 32) gate_warp(p, mode, t_last, floor_, k, ids, off, n_ids, opportunistic);
     if (p.part != BLS_PART_TABLE_RR || mode == BLS_MODE_LOOKUP_ONLY) return;
     __threadfence_block();
     __syncthreads();                                   // the wave plan is visible to the other warps
@@ -138,11 +154,11 @@ __global__ void __launch_bounds__(1024) bls_gate_kernel(BlsParams p, int mode, l
 __global__ void __launch_bounds__(32) bls_commit_kernel(BlsParams p) { commit_lane(p, threadIdx.x); }
 
 void bls_launch_gate(const bls_plan_t *pl, int mode, long long t_last, long long forced_floor, int k,
-                     const int *ids, const int *off, long long n_ids)
+                     const int *ids, const int *off, long long n_ids, int opportunistic)
 {
     // table-wise: one warp per rank for the router's first half (warp 0 is also the gate)
     const bool meta = pl->prm.part == BLS_PART_TABLE_RR && mode != BLS_MODE_LOOKUP_ONLY;
-    bls_gate_kernel<<<1, meta ? 32 * pl->prm.P : 32, 0, pl->stream>>>(pl->prm, mode, t_last, forced_floor, k, ids, off, n_ids);
+    bls_gate_kernel<<<1, meta ? 32 * pl->prm.P : 32, 0, pl->stream>>>(pl->prm, mode, t_last, forced_floor, k, ids, off, n_ids, opportunistic);
 }
 
 void bls_launch_commit(const bls_plan_t *pl)

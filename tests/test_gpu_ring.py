@@ -151,3 +151,42 @@ def test_host_buffer_entry_points():
     for it, (ids, off) in enumerate(inputs):
         want = oracle.pool_definition(P, T, b, w.tables, data, ids, off)
         assert oracle.vector_rel_err(got[it].numpy(), want) <= 1e-5
+
+
+def test_random_delays_are_masked_by_the_bound():
+    """Section V-E setting 2 / Section VI-B: every rank is delayed by a uniform random time
+    before each iteration.  Bound 0 pays the largest of the P delays in every iteration;
+    a bound k > 0 lets ranks drift apart and hides part of it.  Results do not change."""
+    w = bi.tiny_workload(T=4, P=4, b=64, rows=500, dim=16, lengths="poisson10")
+    tabs = dev_tables(w, [bi.table_values(t) for t in w.tables])
+    n_iter, span = 40, 400_000                                  # delays uniform in [0, 400 us]
+    inputs = [bi.make_iteration(w, t) for t in range(n_iter)]
+    d_in = [(torch.from_numpy(i).cuda(), torch.from_numpy(o).cuda()) for i, o in inputs]
+    times, outs = {}, {}
+    for k in (0, 4):
+        plan = make_plan(w, tabs, k)
+        for r in range(w.P):
+            bls.bls_set_random_stall(plan, r, span, seed=1234)
+        bls.bls_set_waves_per_step(plan, w.P + 1)               # one wave per rank that may act, plus the forcing one
+        got = []
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        e0.record()
+        for t in range(n_iter):
+            out, it = bls.bls_step(plan, k, *d_in[t])
+            if out is not None:
+                got.append(out.clone())
+        while True:
+            out, it = bls.bls_drain(plan)
+            if out is None:
+                break
+            got.append(out.clone())
+        e1.record()
+        torch.cuda.synchronize()
+        status, lag = bls.bls_status(plan)
+        assert status == bls.BLS_OK and lag <= k and len(got) == n_iter
+        times[k], outs[k] = e0.elapsed_time(e1) / n_iter, got
+    assert all(torch.equal(a, b) for a, b in zip(outs[0], outs[4]))
+    # bound 0: about the mean of the maximum of four delays (320 us) per iteration
+    assert times[0] > 0.25
+    assert times[4] < 0.9 * times[0], times
