@@ -50,6 +50,8 @@ def parse_args():
                     help="hot rows per table staged in shared memory (0 = off, -1 = the workload's default)")
     ap.add_argument("--delay-us", type=float, default=0.0,
                     help="also time the loop with a uniform random delay in [0, 2*D] us per rank and iteration")
+    ap.add_argument("--straggler", action="store_true",
+                    help="also time the loop with a fixed delay on every rank (the stall-free step time) and twice that on the last rank")
     ap.add_argument("--ks", default="", help="comma-separated bounds to time instead of the workload's own")
     return ap.parse_args()
 
@@ -406,6 +408,21 @@ def run_mine(args):
             bls.bls_set_random_stall(plan, r, 0, 2024)
         delay_sweep["mean_delay_us"] = args.delay_us
         delay_sweep["expected_k0_extra_us"] = 2 * args.delay_us * w.P / (w.P + 1)
+    straggler = None
+    if args.straggler:
+        # every rank is delayed by the stall-free step time before each iteration, the last rank by twice that:
+        # a consistent straggler, which no bound can hide (Section IV, last paragraph)
+        delta_ns = int(by_k[0][0] / args.steps * 1e6)
+        for r in range(w.P):
+            bls.bls_set_stall(plan, r, delta_ns * (2 if r == w.P - 1 else 1))
+        straggler = {"delay_us": delta_ns / 1e3, "last_rank_delay_us": 2 * delta_ns / 1e3}
+        n_s = max(10, args.steps // 4)
+        u_s = float(sum(Ls[t % nd] for t in range(n_s)))
+        for k in ks:
+            ms, _ = aggregate(timed(k, n_s), u_s, world, dev)
+            straggler[str(k)] = {"ms_per_step": ms / n_s}
+        for r in range(w.P):
+            bls.bls_set_stall(plan, r, 0)
     clocks = sampler.stop() if sampler else None
     st, lag = bls.bls_status(plan)
     if st != bls.BLS_OK:
@@ -441,7 +458,7 @@ def run_mine(args):
                      "bytes_per_launch": gather_bytes, "ms_per_launch": ms_gather, "peak_source": peak_src},
         "stage_ms_per_step": {"route": prof["ms_route"] / max(1, prof["calls"]), "gather_pool_return": ms_gather,
                               "ring": prof["ms_ring"] / max(1, prof["calls"])},
-        "clocks": clocks, "e2e": e2e, "gpu_launches": launches, "delay_sweep": delay_sweep,
+        "clocks": clocks, "e2e": e2e, "gpu_launches": launches, "delay_sweep": delay_sweep, "straggler": straggler,
     }
     if not args.no_cpu_baseline and world == 1:
         result["cpu_baseline"] = cpu_baseline(w, inputs)
