@@ -182,7 +182,7 @@ bls_status_t bls_profile_read(bls_plan_t *plan, double *ms_route, double *ms_gat
                               int64_t *calls, int64_t *kernels);
 
 /* Tuning of the gather-pool kernel (results do not depend on it): bags_per_run =
- * consecutive sub-bags one lane group streams (0 = keep; default about 320 rows'
+ * consecutive sub-bags one lane group streams (0 = keep; default about 160 rows'
  * worth), rows_in_flight = row loads per batch, 4 or 8 (0 = keep; default 4). */
 bls_status_t bls_set_tuning(bls_plan_t *plan, int bags_per_run, int rows_in_flight);
 
