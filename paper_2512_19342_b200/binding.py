@@ -104,7 +104,10 @@ class Plan:
     def __del__(self):
         h, self.handle = getattr(self, "handle", None), None
         if h:
-            lib().bls_destroy(h)
+            try:
+                lib().bls_destroy(h)
+            except Exception:          # interpreter shutting down: the process is about to free everything anyway
+                pass
 
 
 def bls_plan_bytes(tables: Sequence[torch.Tensor], part: str, P: int, local_batch: int, k_max: int,

@@ -96,6 +96,12 @@ CASES = [
     ("narrow_rows", lambda: bi.tiny_workload(T=3, P=2, b=257, rows=100, dim=4, lengths="pareto15c")),
     ("dim128_f32", lambda: bi.tiny_workload(T=2, P=2, b=40, rows=300, dim=128, lengths="poisson20c")),
     ("f16_dim8", lambda: bi.tiny_workload(T=5, P=3, b=33, rows=77, dim=8, dtype="f16", lengths="mixed")),
+    ("many_tables", lambda: bi.tiny_workload(T=70, P=3, b=9, rows=40, dim=16, lengths="mixed")),           # > 32 (owner, table) pairs
+    ("max_ranks", lambda: bi.tiny_workload(T=40, P=32, b=5, rows=64, dim=32, lengths="poisson10")),
+    ("max_ranks_rowwise", lambda: bi.tiny_workload(T=3, P=32, b=7, rows=1000, dim=64, dtype="bf16",
+                                                   partition="row_block", lengths="poisson20c")),
+    ("rowwise_more_ranks_than_lanes", lambda: bi.tiny_workload(T=4, P=12, b=20, rows=300, dim=16,
+                                                               partition="row_block", lengths="poisson10")),  # 4 lanes, 12 owners
 ]
 
 

@@ -190,3 +190,16 @@ def test_random_delays_are_masked_by_the_bound():
     # bound 0: about the mean of the maximum of four delays (320 us) per iteration
     assert times[0] > 0.25
     assert times[4] < 0.9 * times[0], times
+
+
+def test_largest_ring():
+    """k_max = 15 (16 slots) and 32 ranks, the limits of a plan."""
+    w = bi.tiny_workload(T=6, P=32, b=3, rows=50, dim=8, lengths="mixed")
+    tabs = dev_tables(w, [bi.table_values(t) for t in w.tables])
+    ref, *_ = run_loop(w, tabs, 0, 20)
+    outs, _, status, lag = run_loop(w, tabs, 15, 20, check_views=True)
+    assert status == bls.BLS_OK and lag == 0
+    assert all(torch.equal(outs[i], ref[i]) for i in range(20))
+    outs, _, status, lag = run_loop(w, tabs, 15, 20, stalls={5: 6_000_000, 31: 1_000_000})   # longer than a host step
+    assert status == bls.BLS_OK and 1 <= lag <= 15
+    assert all(torch.equal(outs[i], ref[i]) for i in range(20))
