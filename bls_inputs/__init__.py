@@ -283,6 +283,8 @@ def _bag_lengths(w: Workload, rng: np.random.Generator, n: int) -> np.ndarray:
     if w.lengths == "pareto15c":
         u = rng.random(n)
         return np.minimum(100, np.floor((1.0 - u) ** (-1.0 / 1.5))).astype(np.int64)
+    if w.lengths == "extremes":                       # empty, single and maximum-length (100) bags
+        return rng.choice(np.array([0, 1, 100]), size=n).astype(np.int64)
     if w.lengths == "mixed":                          # 0..5 with empties, for edge cases
         return rng.integers(0, 6, size=n).astype(np.int64)
     raise ValueError(w.lengths)

@@ -168,6 +168,10 @@ bls_status_t bls_set_random_stall(bls_plan_t *plan, int rank, int64_t max_ns, ui
  * at most P+1): all but the last wait only for the earliest rank that can act, which lets
  * ranks act at different moments and catch up; the last one enforces the bound. */
 bls_status_t bls_set_waves_per_step(bls_plan_t *plan, int waves);
+/* Debug aid: while enabled, the output slot an iteration is issued into is first filled
+ * with 0xFF bytes (NaN), so that a bag that was not written, or a slot read before its data
+ * arrived, shows up in the result.  Costs one pass over the slot per step. */
+bls_status_t bls_set_poison(bls_plan_t *plan, int enable);
 /* Upper limit of any single device-side wait (default 2 s). */
 bls_status_t bls_set_wait_limit(bls_plan_t *plan, int64_t ns);
 

@@ -287,6 +287,16 @@ static void enqueue_wave(bls_plan_t *pl, int mode, long long t_last, long long f
     pl->kernels_launched += 2 + bls_route_kernels(pl);
 }
 
+// Debug aid: a slot that is about to receive iteration `iter` holds an iteration that has
+// been handed back already; filling it with 0xFF bytes (NaN) makes any bag the gather
+// kernel fails to write, and any read of a slot before its data has arrived, visible.
+static void poison_slot(const bls_plan_t *pl, long long iter)
+{
+    if (!pl->poison) return;
+    cudaMemsetAsync(pl->prm.out + (size_t)(iter % pl->prm.S) * pl->prm.out_slot_elems, 0xFF,
+                    sizeof(float) * (size_t)pl->prm.out_slot_elems, pl->stream);
+}
+
 static const float *slot_out(const bls_plan_t *pl, long long iter)
 {
     return pl->prm.out + (size_t)(iter % pl->prm.S) * pl->prm.out_slot_elems;
@@ -297,6 +307,7 @@ bls_status_t bls_route(bls_plan_t *pl, int64_t iter, const int32_t *ids, const i
 {
     if (!pl || !offsets || (!ids && n_ids > 0) || n_ids < 0) return BLS_EINVAL;
     if (iter != pl->t_next || pl->t_handed != pl->t_next || pl->routed_only >= 0) return BLS_ESTATE;
+    poison_slot(pl, iter);
     bls_launch_gate(pl, BLS_MODE_ROUTE_ONLY, iter, -1, 0, ids, offsets, n_ids, 0);
     bls_launch_route(pl);
     bls_launch_commit(pl);
@@ -326,6 +337,7 @@ bls_status_t bls_step(bls_plan_t *pl, int k, const int32_t *ids, const int32_t *
     if (pl->k_cur >= 0 && pl->k_cur != k && pl->t_handed != pl->t_next) return BLS_ESTATE;
     pl->k_cur = k;
     const long long t = pl->t_next++;
+    poison_slot(pl, t);
     // With injected delays the ranks act at different moments: a few opportunistic waves
     // (while the iteration to hand back is incomplete they wait for the earliest rank that can act) let them drift apart and catch
     // up, the last wave enforces the bound.  Without delays one wave does everything.
@@ -478,6 +490,13 @@ bls_status_t bls_set_random_stall(bls_plan_t *pl, int rank, int64_t max_ns, uint
                    cudaStreamSynchronize(pl->stream) == cudaSuccess
                ? BLS_OK
                : BLS_ECUDA;
+}
+
+bls_status_t bls_set_poison(bls_plan_t *pl, int enable)
+{
+    if (!pl) return BLS_EINVAL;
+    pl->poison = enable ? 1 : 0;
+    return BLS_OK;
 }
 
 bls_status_t bls_set_waves_per_step(bls_plan_t *pl, int waves)

@@ -121,6 +121,7 @@ struct bls_plan {
     int rows_in_flight;           // gather kernel: row loads per batch (4 or 8)
     long long *h_rows;            // host copy of the table heights
     int max_waves;                // with injected delays: waves per step (the last one enforces the bound)
+    int poison;                   // debug: fill an output slot with NaN patterns before an iteration is issued into it
     int hot_attached;             // a hot-row buffer has been attached
 };
 #define BLS_PROF_MAX 1024

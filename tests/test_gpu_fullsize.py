@@ -42,6 +42,7 @@ def test_full_size_iteration(num):
     cap = int(np.diff(off[::T * b].astype(np.int64)).max()) + 64
     k = max(w.ks)
     plan = bls.bls_plan(tabs, w.partition, P, b, k, cap)
+    bls.bls_set_poison(plan, True)                     # the slot starts as NaN: every bag must be written
     d_ids, d_off = torch.from_numpy(ids).cuda(), torch.from_numpy(off).cuda()
     out, it = bls.bls_step(plan, k, d_ids, d_off)
     assert (out is None) == (k > 0)
@@ -65,6 +66,6 @@ def test_full_size_iteration(num):
     assert err <= TOL[w.tables[0].dtype], err
     empty = lens[sel] == 0
     assert np.all(got[empty] == 0)
-    # properties that hold at any size: every bag written, totals consistent
+    # properties that hold at any size: every bag written (no NaN left from the poison fill), totals consistent
     assert int(view["sendcounts"].sum()) == len(ids)
     assert torch.isfinite(out).all()

@@ -35,7 +35,9 @@ def make_plan(w, tabs, k_max, cap=None):
             per = np.diff(off[::w.T * w.local_batch].astype(np.int64))
             cap = max(cap, int(per.max()))
         cap = int(cap * 1.25) + 16
-    return bls.bls_plan(tabs, w.partition, w.P, w.local_batch, k_max, cap)
+    plan = bls.bls_plan(tabs, w.partition, w.P, w.local_batch, k_max, cap)
+    bls.bls_set_poison(plan, True)          # every bag must be written: an unwritten one would show up as NaN
+    return plan
 
 
 def check_route(w, view, ids, off):
@@ -96,6 +98,9 @@ CASES = [
     ("narrow_rows", lambda: bi.tiny_workload(T=3, P=2, b=257, rows=100, dim=4, lengths="pareto15c")),
     ("dim128_f32", lambda: bi.tiny_workload(T=2, P=2, b=40, rows=300, dim=128, lengths="poisson20c")),
     ("f16_dim8", lambda: bi.tiny_workload(T=5, P=3, b=33, rows=77, dim=8, dtype="f16", lengths="mixed")),
+    ("extreme_bags", lambda: bi.tiny_workload(T=3, P=2, b=50, rows=300, dim=64, lengths="extremes")),
+    ("extreme_bags_rowwise", lambda: bi.tiny_workload(T=3, P=4, b=50, rows=300, dim=32, dtype="f16",
+                                                      partition="row_block", lengths="extremes")),
     ("many_tables", lambda: bi.tiny_workload(T=70, P=3, b=9, rows=40, dim=16, lengths="mixed")),           # > 32 (owner, table) pairs
     ("max_ranks", lambda: bi.tiny_workload(T=40, P=32, b=5, rows=64, dim=32, lengths="poisson10")),
     ("max_ranks_rowwise", lambda: bi.tiny_workload(T=3, P=32, b=7, rows=1000, dim=64, dtype="bf16",
