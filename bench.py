@@ -52,6 +52,8 @@ def parse_args():
                     help="also time the loop with a uniform random delay in [0, 2*D] us per rank and iteration")
     ap.add_argument("--straggler", action="store_true",
                     help="also time the loop with a fixed delay on every rank (the stall-free step time) and twice that on the last rank")
+    ap.add_argument("--a2a", action="store_true",
+                    help="micro-benchmark of the stand-alone BLS alltoallv (message size and repetition sweeps)")
     ap.add_argument("--ks", default="", help="comma-separated bounds to time instead of the workload's own")
     return ap.parse_args()
 
@@ -465,8 +467,66 @@ def run_mine(args):
     print(json.dumps(result))
 
 
+def run_a2a(args):
+    """Pure-exchange micro-benchmark (the paper's Section V-D): equal-sized alltoallv between 8 logical
+    ranks, time per call against the bytes each rank sends, and back-to-back calls at 32 KB per rank."""
+    import torch
+    import paper_2512_19342_b200 as bls
+    torch.cuda.set_device(0)
+    P = 8
+
+    def request(per_rank):
+        seg = max(1, per_rank // P)
+        counts = torch.full((P, P), seg, dtype=torch.int64, device="cuda")
+        sd = (torch.arange(P, device="cuda", dtype=torch.int64) * seg).repeat(P, 1)
+        send = torch.randint(0, 255, (P, seg * P), dtype=torch.uint8, device="cuda")
+        return send, counts, sd, seg
+
+    def time_calls(a2a, req, n, k):
+        send, counts, sd, seg = req
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        e0.record()
+        out = 0
+        for j in range(n):
+            if j - out > k:                     # more than k requests outstanding: complete the oldest
+                a2a.wait()
+                out += 1
+            a2a.post(send, counts, sd, seg)
+        while out < n:
+            a2a.wait()
+            out += 1
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / n * 1e3    # us per call
+
+    sizes = {}
+    for per_rank in [8, 64, 512, 4096, 32768, 262144, 2097152, 16777216, 134217728, 268435456]:
+        a2a = bls.A2a(P, 0, per_rank + 64)
+        req = request(per_rank)
+        n = 2000 if per_rank <= 262144 else (200 if per_rank <= 16777216 else 20)
+        time_calls(a2a, req, min(n, 20), 0)
+        us = time_calls(a2a, req, n, 0)
+        sizes[str(per_rank)] = {"us_per_call": us, "GB_per_s": 2 * P * (per_rank // P * P) / us / 1e3}
+        assert a2a.status() == bls.BLS_OK
+        del a2a, req
+    reps = {}
+    req = request(32768)
+    for k in (0, 4):
+        a2a = bls.A2a(P, k, 32768 + 64)
+        time_calls(a2a, req, 50, k)
+        reps[str(k)] = {str(n): time_calls(a2a, req, n, k) * n / 1e3 for n in (1, 10, 100, 1000, 10000, 100000)}
+        assert a2a.status() == bls.BLS_OK
+    print(json.dumps({"mode": "a2a", "ranks": P, "by_bytes_per_rank_k0": sizes,
+                      "ms_total_by_repetitions_32KB": reps,
+                      "note": "GB/s counts bytes read plus bytes written; one post kernel and one completion kernel per call"}))
+
+
 def main():
     args = parse_args()
+    if args.a2a:
+        run_a2a(args)
+        return
     if args.impl == "reference":
         run_reference(args)
     else:

@@ -225,6 +225,34 @@ const char *bls_strerror(int status);
 bls_status_t bls_fill_hash_table(void *weight, int64_t rows, int32_t dim, int32_t dtype,
                                  uint64_t seed, int32_t t, void *cuda_stream);
 
+/* ---- the collective on its own: BLS alltoallv of raw bytes (Section III-C) ----
+ * P logical ranks exchange byte segments.  bls_a2a_post initiates request j: rank src's
+ * segment for dst (sendcounts[src][dst] bytes at sendbuf + src*send_stride +
+ * sdispls[src][dst]) is put into dst's receive buffer of slot j mod (k_max+1) at
+ * rdispls[dst][src] = sum of the counts of lower-ranked sources, and the arrival is
+ * counted; nothing waits.  bls_a2a_wait completes the OLDEST outstanding request (it
+ * checks that every receiver counted P messages) and hands out its slot: *recv (device,
+ * rank dst at dst*recv_stride), *recvcounts / *rdispls (device, int64 [P][P] indexed
+ * [dst][src]), valid until k_max+1 further posts.  At most k_max+1 requests may be
+ * outstanding (BLS_ESTATE otherwise): k_max = 0 is a plain alltoallv.
+ *   workspace        device, 256-byte aligned, bls_a2a_bytes() long, borrowed
+ *   sendbuf/sendcounts/sdispls  device; counts and displacements are int64 [P][P] in bytes
+ *   max_segment_bytes host hint: the largest sendcounts entry (sizes the launch)
+ * Asynchronous on the stream; device-detected conditions (segment outside the send
+ * stride: BLS_EINVAL, receive capacity exceeded: BLS_ENOSPC) via bls_a2a_status, which
+ * synchronises. */
+typedef struct bls_a2a bls_a2a_t;
+bls_status_t bls_a2a_bytes(int P, int k_max, int64_t max_bytes_per_rank, size_t *bytes /*host*/);
+bls_status_t bls_a2a_create(int P, int k_max, int64_t max_bytes_per_rank, void *workspace, size_t bytes,
+                            void *cuda_stream, bls_a2a_t **handle /*host out*/);
+void bls_a2a_destroy(bls_a2a_t *handle);
+bls_status_t bls_a2a_post(bls_a2a_t *handle, const void *sendbuf, int64_t send_stride,
+                          const int64_t *sendcounts, const int64_t *sdispls, int64_t max_segment_bytes);
+bls_status_t bls_a2a_wait(bls_a2a_t *handle, const void **recv /*host out*/, int64_t *recv_stride /*host out*/,
+                          const int64_t **recvcounts /*host out*/, const int64_t **rdispls /*host out*/,
+                          int64_t *request /*host out*/);
+bls_status_t bls_a2a_status(bls_a2a_t *handle);
+
 /* ---- allocation-free router (the paper has no counterpart: this entry point
  * exists for deployment reasons only) ----
  * Step (1) for table-wise round-robin placement, for callers that cannot

@@ -25,7 +25,8 @@ EXPORTS = ["bls_plan_bytes", "bls_plan", "bls_destroy", "bls_route", "bls_lookup
            "bls_drain", "bls_step_host", "bls_drain_host", "bls_view", "bls_counters", "bls_status",
            "bls_set_stall", "bls_set_wait_limit", "bls_strerror", "bls_fill_hash_table",
            "bls_profile", "bls_profile_read", "bls_set_tuning", "bls_route_table_rr_static",
-           "bls_set_random_stall", "bls_set_waves_per_step", "bls_set_poison", "bls_hot_bytes", "bls_hot_attach", "bls_hot_observe", "bls_hot_build", "bls_hot_view"]
+           "bls_set_random_stall", "bls_set_waves_per_step", "bls_set_poison", "bls_a2a_bytes", "bls_a2a_create", "bls_a2a_destroy", "bls_a2a_post", "bls_a2a_wait",
+           "bls_a2a_status", "bls_hot_bytes", "bls_hot_attach", "bls_hot_observe", "bls_hot_build", "bls_hot_view"]
 
 
 class BlsError(RuntimeError):
@@ -299,3 +300,54 @@ def bls_hot_view(plan: Plan):
         off = ptr - buf.data_ptr()
         return buf[off:off + 4 * n].view(torch.int32)
     return wrap(rows.value, plan.T * k.value).view(plan.T, k.value), wrap(count.value, plan.T)
+
+
+class A2a:
+    """Handle of a stand-alone BLS alltoallv (raw bytes between the logical ranks)."""
+
+    def __init__(self, P: int, k_max: int, max_bytes_per_rank: int, device="cuda",
+                 stream: Optional[torch.cuda.Stream] = None):
+        n = C.c_size_t(0)
+        _check(lib().bls_a2a_bytes(P, k_max, C.c_int64(max_bytes_per_rank), C.byref(n)), "bls_a2a_bytes")
+        ws = torch.empty(n.value + 256, dtype=torch.uint8, device=device)
+        pad = (-ws.data_ptr()) % 256
+        self.workspace = ws[pad:pad + n.value]
+        self.P, self.k_max = P, k_max
+        self.handle = C.c_void_p()
+        _check(lib().bls_a2a_create(P, k_max, C.c_int64(max_bytes_per_rank), C.c_void_p(self.workspace.data_ptr()),
+                                    C.c_size_t(n.value), _stream_ptr(stream), C.byref(self.handle)), "bls_a2a_create")
+        self._keep = []
+
+    def post(self, sendbuf: torch.Tensor, sendcounts: torch.Tensor, sdispls: torch.Tensor, max_segment_bytes: int):
+        """sendbuf uint8 [P][stride]; sendcounts/sdispls int64 [P][P] (bytes), all on the device."""
+        self._keep.append((sendbuf, sendcounts, sdispls))
+        del self._keep[:-(self.k_max + 2)]
+        _check(lib().bls_a2a_post(self.handle, C.c_void_p(sendbuf.data_ptr()), C.c_int64(sendbuf.shape[1]),
+                                  C.c_void_p(sendcounts.data_ptr()), C.c_void_p(sdispls.data_ptr()),
+                                  C.c_int64(max_segment_bytes)), "bls_a2a_post")
+
+    def wait(self):
+        """Completes the oldest request: (recv uint8 [P][stride], recvcounts, rdispls int64 [P][P], request number)."""
+        recv, rc, rd = C.c_void_p(), C.c_void_p(), C.c_void_p()
+        stride, req = C.c_int64(0), C.c_int64(-1)
+        _check(lib().bls_a2a_wait(self.handle, C.byref(recv), C.byref(stride), C.byref(rc), C.byref(rd), C.byref(req)),
+               "bls_a2a_wait")
+        ws, P = self.workspace, self.P
+
+        def view(ptr, nbytes):
+            off = ptr - ws.data_ptr()
+            return ws[off:off + nbytes]
+        return (view(recv.value, P * stride.value).view(P, stride.value),
+                view(rc.value, 8 * P * P).view(torch.int64).view(P, P),
+                view(rd.value, 8 * P * P).view(torch.int64).view(P, P), req.value)
+
+    def status(self) -> int:
+        return lib().bls_a2a_status(self.handle)
+
+    def __del__(self):
+        h, self.handle = getattr(self, "handle", None), None
+        if h:
+            try:
+                lib().bls_a2a_destroy(h)
+            except Exception:
+                pass
