@@ -197,7 +197,7 @@ def cpu_baseline(w, inputs, target_s=12.0):
     t0 = time.perf_counter()
     oracle_iteration(w, data, ids, off, cores)
     t1 = time.perf_counter() - t0
-    n = int(max(1, min(len(inputs) * 4, round(target_s / max(t1, 1e-3)))))
+    n = int(max(1, min(400, round(target_s / max(t1, 1e-3)))))
     lookups = 0
     t0 = time.perf_counter()
     for i in range(n):

@@ -186,8 +186,8 @@ bls_status_t bls_profile_read(bls_plan_t *plan, double *ms_route, double *ms_gat
                               int64_t *calls, int64_t *kernels);
 
 /* Tuning of the gather-pool kernel (results do not depend on it): bags_per_run =
- * consecutive sub-bags one lane group streams (0 = keep; default about 160 rows'
- * worth), rows_in_flight = row loads per batch, 4 or 8 (0 = keep; default 4). */
+ * consecutive sub-bags one lane group streams (0 = keep; default 4 to 24, about 160 rows'
+ * worth for table-wise and 50 for row-wise placement), rows_in_flight = row loads per batch, 4 or 8 (0 = keep; default 4). */
 bls_status_t bls_set_tuning(bls_plan_t *plan, int bags_per_run, int rows_in_flight);
 
 /* ---- hot-row staging (optional; table-wise placement only) ----
