@@ -54,6 +54,8 @@ def parse_args():
                     help="also time the loop with a fixed delay on every rank (the stall-free step time) and twice that on the last rank")
     ap.add_argument("--a2a", action="store_true",
                     help="micro-benchmark of the stand-alone BLS alltoallv (message size and repetition sweeps)")
+    ap.add_argument("--uniform-ids", action="store_true",
+                    help="draw IDs uniformly instead of from the workload's Zipf law (no hot rows: every row read goes to DRAM)")
     ap.add_argument("--ks", default="", help="comma-separated bounds to time instead of the workload's own")
     return ap.parse_args()
 
@@ -291,6 +293,8 @@ def select(w, args):
         w = dataclasses.replace(w, tables=w.tables[:args.tables], name=f"{w.name}_first{args.tables}tables")
     if args.ks:
         w = dataclasses.replace(w, ks=tuple(int(x) for x in args.ks.split(",")))
+    if args.uniform_ids:
+        w = dataclasses.replace(w, id_dist="uniform", name=f"{w.name}_uniform_ids")
     return w
 
 
