@@ -52,7 +52,7 @@ typedef enum {
 
 typedef enum { BLS_F32 = 0, BLS_BF16 = 1, BLS_F16 = 2 } bls_dtype_t;
 
-/* Table placement ("a given partitioning strategy", Section I):
+/* Table placement (Section I leaves the partitioning strategy open):
  *   TABLE_RR   owner(t, id) = t mod P, owner-local row = id
  *   ROW_BLOCK  owner(t, id) = id / ceil(rows_t / P), owner-local row = id - owner*ceil(rows_t/P) */
 typedef enum { BLS_PART_TABLE_RR = 0, BLS_PART_ROW_BLOCK = 1 } bls_part_t;

@@ -11,7 +11,7 @@
  * What it states (paper passages in brackets):
  *   - batch row-block partition: sample g of the global batch belongs to
  *     requester rank g / b                                    [Section I, par. 6]
- *   - tables are distributed "by a given partitioning strategy"; the two used
+ *   - the paper leaves the table partitioning strategy open; the two used
  *     here are table-wise round-robin (owner = t mod P) and row-wise blocks
  *     (owner = id / ceil(N_t / P))                            [Section I, par. 6]
  *   - every rank determines the vector IDs it needs from every other rank and

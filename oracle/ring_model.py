@@ -3,7 +3,7 @@
 P ranks exchange one request message and one response message per iteration.
 Iteration j lives in slot j mod (k+1).  Three monotone counters per rank record
 progress (Section III-C: tagged puts are counted per iteration; Section IV,
-Listing 2: a rank may run ahead until ``unfinished > bound``, completion is FIFO,
+Listing 2: a rank may run ahead until more than k requests are outstanding, completion is FIFO,
 and the last batch drains everything):
 
   posted[r]  iterations whose requests rank r has put into all owners' slots
@@ -11,7 +11,7 @@ and the last batch drains everything):
   done[r]    iterations rank r has completed (oldest first)
 
 Enabling rules (reading of Section III-D and Listing 2's comment that a rank too
-far ahead "will overwrite buffer"):
+far ahead would overwrite a buffer that is still in use):
   post(r, j)    needs min over ranks of done >= j - k      (slot j mod S is free)
   serve(o, j)   needs every rank to have posted j          (all P sources, self included)
   consume(r, j) needs every owner to have served j         (all P messages with that tag)

@@ -5,8 +5,8 @@
 // Reading of the paper (Section III-C, III-D, Section IV / Listing 2):
 //   * iteration j uses slot j mod S, S = k_max + 1 buffers created at plan time;
 //   * a rank may put the requests of iteration j only when every rank has
-//     completed iteration j - k - 1, i.e. min(done) >= j - k (otherwise it
-//     "will overwrite buffer", Listing 2);
+//     completed iteration j - k - 1, i.e. min(done) >= j - k (Listing 2 notes that a
+//     rank too far ahead would overwrite a buffer);
 //   * an owner answers iteration j once all P sources have posted it (tagged
 //     messages are counted per iteration);
 //   * a rank completes iteration j once all owners have answered it; completion

@@ -1,6 +1,6 @@
 // Step 1, the router: every requester rank sorts the rows it needs by owner rank
-// (Section I: "each process determines the vector IDs required from other
-// processes, and retrieves them through an alltoallv").  Output per requester:
+// (Section I: every rank works out which vector IDs it needs from which other rank and
+// fetches them with an alltoallv).  Output per requester:
 // sendcounts / sdispls, the stably packed send buffer of owner-local rows, and
 // the start of every sub-bag inside it (the owner rebuilds bag boundaries from
 // consecutive differences).

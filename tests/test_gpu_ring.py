@@ -1,5 +1,5 @@
 """The BLS slot ring on the GPU: output for any bound k equals the synchronous
-output (Abstract: accuracy is fully preserved; Section III-D: k = 0 is the plain
+output (Abstract: the bound does not change what is computed; Section III-D: k = 0 is the plain
 alltoallv), ranks really lag under injected delays, never by more than k, and a
 wait that cannot end in time returns a status instead of hanging.  GPU only."""
 import numpy as np

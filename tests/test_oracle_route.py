@@ -3,7 +3,7 @@
 Each test fixes the oracle to something other than itself: a hand-enumerated
 fixture, a closed form the paper states, or a library routine (numpy's stable
 argsort and cumsum) that *is* the textbook alltoallv of bound k = 0
-(Section III-D: "semantically equivalent to MPI_Alltoallv").
+(Section III-D: with a zero bound the collective has the semantics of MPI_Alltoallv).
 """
 import json
 import os
