@@ -141,7 +141,10 @@ bls_status_t bls_drain(bls_plan_t *plan, const float **out /*host out*/, int64_t
 /* The same two calls with HOST input and output buffers: ids/offsets are copied
  * to a staging area of the ring (pinned memory recommended), and the iteration
  * handed back, if any, is copied to host_out (fp32 [P][b][T][dim]; may be NULL to
- * skip the copy).  Copies are asynchronous on the plan's stream. */
+ * skip the copy).  The copies run asynchronously on two internal streams (upload of the
+ * next iteration and download of the previous result overlap); the plan's stream waits for
+ * them, so synchronising it, or enqueuing work on it, after the call sees host_out complete.
+ * The host buffers must stay untouched until then. */
 bls_status_t bls_step_host(bls_plan_t *plan, int k, const int32_t *ids /*host*/,
                            const int32_t *offsets /*host*/, int64_t n_ids,
                            float *host_out /*host*/, int64_t *out_iter /*host out*/);

@@ -228,6 +228,13 @@ void bls_destroy(bls_plan_t *plan)
         for (int i = 0; i < BLS_PROF_MAX * 4; i++) cudaEventDestroy(plan->prof_ev[i]);
         free(plan->prof_ev);
     }
+    if (plan->host_path) {
+        cudaStreamDestroy(plan->s_in);
+        cudaStreamDestroy(plan->s_out);
+        cudaEventDestroy(plan->e_in);
+        cudaEventDestroy(plan->e_comp);
+        cudaEventDestroy(plan->e_out);
+    }
     free(plan->h_rows);
     free(plan);
 }
@@ -381,41 +388,73 @@ bls_status_t bls_drain(bls_plan_t *pl, const float **out, int64_t *out_iter)
     return launch_check();
 }
 
+// Host-buffer path: the copies run on two streams of their own so that the upload of the
+// next iteration and the download of the previous result overlap (PCIe is full duplex) and
+// only the kernels sit between them.  The plan's stream waits for both, so work enqueued
+// on it afterwards, and a synchronisation of it, see the copies complete.
+static bool host_path_ready(bls_plan_t *pl)
+{
+    if (pl->host_path) return true;
+    if (cudaStreamCreateWithFlags(&pl->s_in, cudaStreamNonBlocking) != cudaSuccess ||
+        cudaStreamCreateWithFlags(&pl->s_out, cudaStreamNonBlocking) != cudaSuccess ||
+        cudaEventCreateWithFlags(&pl->e_in, cudaEventDisableTiming) != cudaSuccess ||
+        cudaEventCreateWithFlags(&pl->e_comp, cudaEventDisableTiming) != cudaSuccess ||
+        cudaEventCreateWithFlags(&pl->e_out, cudaEventDisableTiming) != cudaSuccess)
+        return false;
+    // nothing has been enqueued on the copy streams yet: order them after what the plan's stream holds
+    if (cudaEventRecord(pl->e_comp, pl->stream) != cudaSuccess) return false;
+    pl->host_path = 1;
+    return true;
+}
+
+static bls_status_t download(bls_plan_t *pl, const float *out, float *host_out)
+{
+    if (cudaEventRecord(pl->e_comp, pl->stream) != cudaSuccess) return BLS_ECUDA;
+    if (out && host_out) {
+        if (cudaStreamWaitEvent(pl->s_out, pl->e_comp, 0) != cudaSuccess ||
+            cudaMemcpyAsync(host_out, out, sizeof(float) * (size_t)pl->prm.out_slot_elems, cudaMemcpyDeviceToHost,
+                            pl->s_out) != cudaSuccess ||
+            cudaEventRecord(pl->e_out, pl->s_out) != cudaSuccess ||
+            cudaStreamWaitEvent(pl->stream, pl->e_out, 0) != cudaSuccess)
+            return BLS_ECUDA;
+    }
+    return BLS_OK;
+}
+
 bls_status_t bls_step_host(bls_plan_t *pl, int k, const int32_t *ids, const int32_t *offsets,
                            int64_t n_ids, float *host_out, int64_t *out_iter)
 {
     if (!pl || !offsets || (!ids && n_ids > 0) || n_ids < 0 || !out_iter) return BLS_EINVAL;
     const BlsParams &p = pl->prm;
     if (n_ids > (long long)p.P * p.cap) return BLS_ENOSPC;
+    if (k < 0 || k > pl->k_max || pl->routed_only >= 0) return BLS_ESTATE;
+    if (!host_path_ready(pl)) return BLS_ECUDA;
     const int slot = (int)(pl->t_next % p.S);
     const size_t G1 = (size_t)p.P * p.T * p.b + 1;
     int *d_ids = p.stage_ids + (size_t)slot * p.P * p.cap;
     int *d_off = p.stage_off + (size_t)slot * G1;
-    if (cudaMemcpyAsync(d_off, offsets, sizeof(int) * G1, cudaMemcpyHostToDevice, pl->stream) != cudaSuccess ||
+    // upload after the previous step's kernels (the staging slot's last user finished long before them)
+    if (cudaStreamWaitEvent(pl->s_in, pl->e_comp, 0) != cudaSuccess ||
+        cudaMemcpyAsync(d_off, offsets, sizeof(int) * G1, cudaMemcpyHostToDevice, pl->s_in) != cudaSuccess ||
         (n_ids > 0 &&
-         cudaMemcpyAsync(d_ids, ids, sizeof(int) * (size_t)n_ids, cudaMemcpyHostToDevice, pl->stream) != cudaSuccess))
+         cudaMemcpyAsync(d_ids, ids, sizeof(int) * (size_t)n_ids, cudaMemcpyHostToDevice, pl->s_in) != cudaSuccess) ||
+        cudaEventRecord(pl->e_in, pl->s_in) != cudaSuccess ||
+        cudaStreamWaitEvent(pl->stream, pl->e_in, 0) != cudaSuccess)
         return BLS_ECUDA;
     const float *out = nullptr;
     bls_status_t st = bls_step(pl, k, d_ids, d_off, n_ids, &out, out_iter);
     if (st != BLS_OK) return st;
-    if (out && host_out &&
-        cudaMemcpyAsync(host_out, out, sizeof(float) * (size_t)p.out_slot_elems, cudaMemcpyDeviceToHost,
-                        pl->stream) != cudaSuccess)
-        return BLS_ECUDA;
-    return BLS_OK;
+    return download(pl, out, host_out);
 }
 
 bls_status_t bls_drain_host(bls_plan_t *pl, float *host_out, int64_t *out_iter)
 {
     if (!pl || !out_iter) return BLS_EINVAL;
+    if (!host_path_ready(pl)) return BLS_ECUDA;
     const float *out = nullptr;
     bls_status_t st = bls_drain(pl, &out, out_iter);
     if (st != BLS_OK) return st;
-    if (out && host_out &&
-        cudaMemcpyAsync(host_out, out, sizeof(float) * (size_t)pl->prm.out_slot_elems,
-                        cudaMemcpyDeviceToHost, pl->stream) != cudaSuccess)
-        return BLS_ECUDA;
-    return BLS_OK;
+    return download(pl, out, host_out);
 }
 
 bls_status_t bls_view(bls_plan_t *pl, int64_t iter, bls_route_view_t *v)

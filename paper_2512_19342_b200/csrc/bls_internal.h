@@ -115,6 +115,10 @@ struct bls_plan {
     int prof_on;
     int prof_n;
     cudaEvent_t *prof_ev;
+    // host-buffer entry points: copy streams and events, created on first use
+    cudaStream_t s_in, s_out;
+    cudaEvent_t e_in, e_comp, e_out;
+    int host_path;
     long long kernels_launched;   // total kernels enqueued through this plan
     int any_stall;                // a delay was injected at some point: ranks may be out of lockstep
     int bags_per_run;             // gather kernel: consecutive sub-bags streamed by one lane group
