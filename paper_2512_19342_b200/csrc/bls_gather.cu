@@ -489,13 +489,14 @@ static void launch_gather(const bls_plan_t *pl)
     const long long bags = (long long)(rowwise ? p.T : p.NI) * p.P * p.b;
     const long long resident_groups = (long long)pl->sm_count * 24 * (32 / LANES);
     long long fit = bags / (2 * resident_groups);
-    const int R = (int)(fit < 1 ? 1 : (fit < pl->bags_per_run ? fit : pl->bags_per_run));
+    int R = (int)(fit < 1 ? 1 : (fit < pl->bags_per_run ? fit : pl->bags_per_run));
+    while ((long long)(rowwise ? p.T : p.NI) * p.P * ((p.b + R - 1) / R) > 0x7fffffffLL) R *= 2;   // run numbers are 32-bit
     const int rpc = (p.b + R - 1) / R;
     // table-wise: runs of sub-bags of one (owner, table, requester); row-wise: runs of bags of one (table, requester)
     const long long n_runs = (long long)(rowwise ? p.T : p.NI) * p.P * rpc;
-    // more blocks than fit at once (late ones find the counter exhausted), fewer for small workloads
+    // persistent blocks: as many as stay resident (3 per SM at 80 registers), fewer for small workloads
     const long long want = (n_runs + 8 * (32 / LANES) - 1) / (8 * (32 / LANES));
-    const int blocks = (int)(want < 1 ? 1 : (want > pl->sm_count * 8 ? pl->sm_count * 8 : want));
+    const int blocks = (int)(want < 1 ? 1 : (want > pl->sm_count * 3 ? pl->sm_count * 3 : want));
     if (rowwise) {
         bls_gather_rowwise_kernel<LANES, DT><<<blocks, 256, 0, pl->stream>>>(p, R, rpc, (int)n_runs);
     } else if (p.hot.enabled) {
