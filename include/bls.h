@@ -103,13 +103,14 @@ bls_status_t bls_plan_bytes(const bls_table_t *tables /*host*/, int T, int part,
 
 /* Build a plan inside `workspace` (device, 256-byte aligned, `bytes` long, borrowed
  * until bls_destroy).  Enqueues the initialisation of counters and descriptors on
- * `cuda_stream` (a cudaStream_t; NULL = default stream).  P <= 32, k_max <= 15, and
- * T <= 3000 for table-wise placement. */
+ * `cuda_stream` (a cudaStream_t; NULL = default stream).  P <= 32, k_max <= 15. */
 bls_status_t bls_plan(const bls_table_t *tables /*host*/, int T, int part, int P, int local_batch,
                       int k_max, int64_t max_ids_per_rank, void *workspace, size_t bytes,
                       void *cuda_stream, bls_plan_t **plan /*host out*/);
 
-void bls_destroy(bls_plan_t *plan);          /* frees host memory only; does not synchronise */
+void bls_destroy(bls_plan_t *plan);          /* frees host-side state (incl. the copy streams and timing
+                                                events it created); the workspace stays the caller's;
+                                                does not synchronise */
 
 /* ---- the synchronous decomposition (bound 0 == plain alltoallv, Section III-D) ----
  * bls_route:  step (1) for every rank for iteration `iter` (must be the next
@@ -168,8 +169,9 @@ bls_status_t bls_set_stall(bls_plan_t *plan, int rank, int64_t ns);
  * can be repeated).  The seed is shared by all ranks of the plan. */
 bls_status_t bls_set_random_stall(bls_plan_t *plan, int rank, int64_t max_ns, uint64_t seed);
 /* While delays are injected, one bls_step runs up to `waves` waves of kernels (default 4,
- * at most P+1): all but the last wait only for the earliest rank that can act, which lets
- * ranks act at different moments and catch up; the last one enforces the bound. */
+ * at most P+1): while the iteration to hand back is still incomplete, a wave waits for the
+ * earliest rank that can act (not for all of them), so ranks act at different moments and
+ * faster ones run ahead; once it is complete waves do not wait; the last wave enforces the bound. */
 bls_status_t bls_set_waves_per_step(bls_plan_t *plan, int waves);
 /* Debug aid: while enabled, the output slot an iteration is issued into is first filled
  * with 0xFF bytes (NaN), so that a bag that was not written, or a slot read before its data
@@ -182,15 +184,17 @@ bls_status_t bls_set_wait_limit(bls_plan_t *plan, int64_t ns);
  * bls_step/bls_drain records events around its three stages (up to 1024 calls
  * are kept).  bls_profile_read synchronises the stream, adds up the recorded
  * calls into milliseconds per stage (gate + router kernels, the gather-pool-return
- * kernel including the commit done by its last block, anything after it), reports how many calls were summed and how
- * many kernels they launched, and clears the record.  Any pointer may be NULL. */
+ * kernel including the commit done by its last block, anything after it), reports how
+ * many calls were summed and how many kernels the plan has launched so far, and clears
+ * the record.  Any pointer may be NULL. */
 bls_status_t bls_profile(bls_plan_t *plan, int enable);
 bls_status_t bls_profile_read(bls_plan_t *plan, double *ms_route, double *ms_gather, double *ms_ring,
                               int64_t *calls, int64_t *kernels);
 
 /* Tuning of the gather-pool kernel (results do not depend on it): bags_per_run =
  * consecutive sub-bags one lane group streams (0 = keep; default 4 to 24, about 160 rows'
- * worth for table-wise and 50 for row-wise placement), rows_in_flight = row loads per batch, 4 or 8 (0 = keep; default 4). */
+ * worth for table-wise and 50 for row-wise placement), rows_in_flight = row loads per
+ * batch, 4 or 8 (0 = keep; default 4). */
 bls_status_t bls_set_tuning(bls_plan_t *plan, int bags_per_run, int rows_in_flight);
 
 /* ---- hot-row staging (optional; table-wise placement only) ----
