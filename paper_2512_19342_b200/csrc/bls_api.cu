@@ -48,7 +48,17 @@ void fill_params(BlsParams &p, const bls_table_t *tables, int T, int part, int P
     p.NI = part == BLS_PART_TABLE_RR ? T : T * P;
     p.NQ = p.NI * b;
     p.cap = (int)((cap + 3) / 4 * 4);          // every rank's send buffer starts on a 16-byte boundary
-    p.tiles_per_table = (b + BLS_ROUTE_TB - 1) / BLS_ROUTE_TB;
+    // Routing tiles.  Row-wise: BLS_ROUTE_TB bags (the scatter kernel's shared-memory tile).
+    // Table-wise: a tile is only copied, so it grows for short bags until a block moves
+    // about 4096 IDs, as long as enough tiles remain to fill the GPU.
+    p.tile_bags = BLS_ROUTE_TB;
+    if (part == BLS_PART_TABLE_RR) {
+        const double avg = (double)cap / ((double)p.NI * b);
+        while (p.tile_bags < b && p.tile_bags * avg < 4096.0 &&
+               (long long)T * P * ((b + 2 * p.tile_bags - 1) / (2 * p.tile_bags)) >= 2048)
+            p.tile_bags *= 2;
+    }
+    p.tiles_per_table = (b + p.tile_bags - 1) / p.tile_bags;
     p.NT = T * p.tiles_per_table;
     // table-wise: NQ starts + 1 terminal entry; row-wise (bag-major): NQ starts + P terminal entries
     p.sub_stride = (long long)align_up((size_t)p.NQ + (part == BLS_PART_TABLE_RR ? 1 : P), 4);

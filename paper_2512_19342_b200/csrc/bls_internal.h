@@ -80,8 +80,9 @@ struct BlsParams {
     int NI;                 // number of (owner, table) pairs
     int NQ;                 // sub-bags per requester = NI * b
     int cap;                // IDs per rank per iteration (send buffer capacity)
-    int NT;                 // routing tiles per requester = T * ceil(b / TB)
-    int tiles_per_table;    // ceil(b / TB)
+    int NT;                 // routing tiles per requester = T * tiles_per_table
+    int tiles_per_table;    // ceil(b / tile_bags)
+    int tile_bags;          // bags per routing tile: BLS_ROUTE_TB row-wise, a multiple of it table-wise
     int row_bytes;
     BlsDev *dev;
     const BlsTableDesc *tab;     // [T]

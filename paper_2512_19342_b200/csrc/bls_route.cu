@@ -18,17 +18,18 @@
 // First half (chunk lengths, scan, counts, displacements): tw_meta_warp, run by the
 // gate kernel.  Second half, here: move every ID to its place and write the sub-bag
 // starts.
-// grid (NT, P): tile = 128 bags of one (requester, table) chunk.  Copies the
-// chunk's IDs to their place in the send buffer (coalesced) and writes the
-// sub-bag starts.
+// grid (NT, P): tile = p.tile_bags bags of one (requester, table) chunk (128 for long
+// bags, up to the whole chunk for short ones, so that a block always has a few
+// thousand IDs to move).  Copies the tile's IDs to their place in the send buffer
+// (coalesced) and writes the sub-bag starts.
 __global__ void __launch_bounds__(256) bls_tw_copy_kernel(BlsParams p)
 {
     const int src = blockIdx.y;
     RouteCtx c;
     if (!route_ctx(p, src, c)) return;
     const int i = blockIdx.x / p.tiles_per_table;
-    const int s0 = (blockIdx.x % p.tiles_per_table) * BLS_ROUTE_TB;
-    const int nb = min(BLS_ROUTE_TB, p.b - s0);
+    const int s0 = (blockIdx.x % p.tiles_per_table) * p.tile_bags;
+    const int nb = min(p.tile_bags, p.b - s0);
     const int t = p.pair[i].t;
     const long long g0 = ((long long)src * p.T + t) * p.b;
     const int *cbp = p.chunk_base + (size_t)src * (p.NI + 1);
@@ -36,13 +37,13 @@ __global__ void __launch_bounds__(256) bls_tw_copy_kernel(BlsParams p)
     const int cn = cbp[i + 1] - cb;              // chunk length accepted by the meta kernel
     const long long off0 = c.off[g0];
     __shared__ int s_lo, s_hi;
-    if (threadIdx.x < nb) {
+    for (int s = threadIdx.x; s < nb; s += blockDim.x) {
         int st, en;
-        if (!bag_range(c, g0 + s0 + threadIdx.x, off0, cn, st, en)) flag(p, BLS_ST_EINVAL);
+        if (!bag_range(c, g0 + s0 + s, off0, cn, st, en)) flag(p, BLS_ST_EINVAL);
         int pos = cb + st;
-        c.sub_start[(size_t)i * p.b + s0 + threadIdx.x] = pos > p.cap ? p.cap : pos;
-        if (threadIdx.x == 0) s_lo = st;
-        if (threadIdx.x == nb - 1) s_hi = en;
+        c.sub_start[(size_t)i * p.b + s0 + s] = pos > p.cap ? p.cap : pos;
+        if (s == 0) s_lo = st;
+        if (s == nb - 1) s_hi = en;
     }
     __syncthreads();
     const unsigned rows = (unsigned)p.tab[t].rows;
@@ -95,56 +96,66 @@ __device__ __forceinline__ int owner_of_row(unsigned id, int blk, unsigned magic
     return (int)q;
 }
 
-// A tile (128 bags of one table of one requester) is routed only if all its bags are
-// well-formed; otherwise it is treated as empty and BLS_EINVAL is latched.  Returns the
-// tile's ID range [lo, hi).
-__device__ __forceinline__ bool tile_range(const BlsParams &p, const RouteCtx &c, long long g0, int nb, int &lo, int &hi)
+// Range of lookups [lo, hi) of a tile (BLS_ROUTE_TB bags of one table of one requester).
+// A tile whose ends are not ordered or leave the ID array is treated as empty and
+// BLS_EINVAL is latched; both row-wise kernels apply the same rule, so the counts
+// and the positions derived from them always agree.
+__device__ __forceinline__ void tile_ends(const BlsParams &p, const RouteCtx &c, long long g0, int nb, int &lo, int &hi)
 {
-    bool ok = true;
-    if ((int)threadIdx.x < nb) {
-        const long long a = c.off[g0 + threadIdx.x], e = c.off[g0 + threadIdx.x + 1];
-        ok = a >= 0 && a <= e && e <= c.n_ids;
-    }
-    ok = __syncthreads_and(ok);
-    if (!ok) { if (threadIdx.x == 0) flag(p, BLS_ST_EINVAL); lo = hi = 0; return false; }
-    lo = c.off[g0];
-    hi = c.off[g0 + nb];
-    return true;
+    const long long a = c.off[g0], e = c.off[g0 + nb];
+    if (a >= 0 && a <= e && e <= c.n_ids) { lo = (int)a; hi = (int)e; return; }
+    flag(p, BLS_ST_EINVAL);
+    lo = hi = 0;
 }
 
-// grid (NT, P): per-tile histogram over destinations, one thread per lookup (coalesced);
-// lanes with the same destination are counted together.
-__global__ void __launch_bounds__(BLS_ROUTE_TB) bls_rw_count_kernel(BlsParams p)
+// grid (NT, P), 128 threads: per-tile histogram over destinations.  All of a thread's
+// IDs are requested before the first one is used; lanes with the same destination are
+// counted together (one shared-memory atomic per distinct destination and warp step).
+#define BLS_RW_PER_THREAD 16
+__global__ void __launch_bounds__(BLS_ROUTE_TB, 10) bls_rw_count_kernel(BlsParams p)
 {
     __shared__ int cnt[BLS_MAX_RANKS];
     const int src = blockIdx.y;
     RouteCtx c;
     if (!route_ctx(p, src, c)) return;
+    const int tid = threadIdx.x, lane = tid & 31;
     const int t = blockIdx.x / p.tiles_per_table;
-    const int s0 = (blockIdx.x % p.tiles_per_table) * BLS_ROUTE_TB;
+    const int s0 = (blockIdx.x - t * p.tiles_per_table) * BLS_ROUTE_TB;
     const int nb = min(BLS_ROUTE_TB, p.b - s0);
-    if (threadIdx.x < BLS_MAX_RANKS) cnt[threadIdx.x] = 0;
+    if (tid < BLS_MAX_RANKS) cnt[tid] = 0;
     int lo, hi;
-    tile_range(p, c, ((long long)src * p.T + t) * p.b + s0, nb, lo, hi);      // contains a barrier
+    tile_ends(p, c, ((long long)src * p.T + t) * p.b + s0, nb, lo, hi);
     const unsigned rows = (unsigned)p.tab[t].rows;
     const int blk = p.tab[t].blk;
     const unsigned magic = p.tab[t].magic;
-    const int lane = threadIdx.x & 31;
-    for (int l0 = lo + (threadIdx.x & ~31); l0 < hi; l0 += BLS_ROUTE_TB) {
-        const int l = l0 + lane;
-        int d = 64 + lane;                                  // no lookup: matches nobody
-        if (l < hi) {
-            unsigned id = (unsigned)__ldcs(c.ids + l);
-            if (id >= rows) { id = 0; flag(p, BLS_ST_ERANGE); }
-            int local;
-            d = owner_of_row(id, blk, magic, local);
-        }
-        const unsigned same = __match_any_sync(0xffffffffu, d);
-        if (l < hi && lane == __ffs(same) - 1) atomicAdd(&cnt[d], __popc(same));
-    }
     __syncthreads();
-    if (threadIdx.x < p.P)
-        p.tile_cnt[((size_t)src * p.NT + blockIdx.x) * p.P + threadIdx.x] = cnt[threadIdx.x];
+    bool bad = false;
+    for (int l0 = lo; l0 < hi; l0 += BLS_RW_PER_THREAD * BLS_ROUTE_TB) {
+        int idr[BLS_RW_PER_THREAD];
+        #pragma unroll
+        for (int q = 0; q < BLS_RW_PER_THREAD; q++) {
+            const int l = l0 + q * BLS_ROUTE_TB + tid;
+            idr[q] = l < hi ? __ldcs(c.ids + l) : 0;
+        }
+        #pragma unroll
+        for (int q = 0; q < BLS_RW_PER_THREAD; q++) {
+            const int l = l0 + q * BLS_ROUTE_TB + tid;
+            if (l - lane < hi) {                            // same for the whole warp
+                int d = 64 + lane;                          // no lookup: matches nobody
+                if (l < hi) {
+                    unsigned id = (unsigned)idr[q];
+                    if (id >= rows) { id = 0; bad = true; }
+                    int local;
+                    d = owner_of_row(id, blk, magic, local);
+                }
+                const unsigned same = __match_any_sync(0xffffffffu, d);
+                if (l < hi && lane == __ffs(same) - 1) atomicAdd(&cnt[d], __popc(same));
+            }
+        }
+    }
+    if (bad) flag(p, BLS_ST_ERANGE);
+    __syncthreads();
+    if (tid < p.P) p.tile_cnt[((size_t)src * p.NT + blockIdx.x) * p.P + tid] = cnt[tid];
 }
 
 // One block per requester: exclusive scan of the tile counts in (destination, tile)
@@ -177,9 +188,6 @@ __global__ void __launch_bounds__(1024) bls_rw_scan_kernel(BlsParams p)
         const int d = threadIdx.x;
         c.sdispls[d] = (int)min(disp[d], (long long)0x7fffffff);
         c.sendcounts[d] = (int)tot[d];
-        // sub-bag starts are kept bag-major [table][sample][dst]: the entry after the last bag
-        // closes every destination's region
-        c.sub_start[(size_t)p.T * p.b * p.P + d] = (int)min(disp[d + 1], (long long)p.cap);
     }
     for (int d = w; d < p.P; d += 32) {
         long long run = disp[d];
@@ -205,103 +213,128 @@ __global__ void __launch_bounds__(1024) bls_rw_scan_kernel(BlsParams p)
     }
 }
 
-// grid (NT, P), one thread per bag.  Inside a tile, the lookups of one
-// destination keep their original order: position = tile base + number of
-// same-destination lookups in earlier bags of the tile + rank inside the bag.
-// The tile's IDs are first staged in shared memory (coalesced) with their owner
-// already computed, so the two per-bag passes run out of shared memory.
-#define BLS_RW_STAGE 2048
-__global__ void __launch_bounds__(BLS_ROUTE_TB) bls_rw_scatter_kernel(BlsParams p)
+// grid (NT, P), 128 threads: places the lookups of one tile and writes its sub-bag starts.
+// The tile's lookups are classified BLS_RW_CHUNK at a time, one thread per lookup
+// (coalesced).  For every destination d a bit mask over the chunk's lookups is built
+// from warp matches (bit i set: lookup i goes to d) together with the number of set bits
+// before each 32-bit word.  Everything else is a rank query on those masks:
+//   position of lookup i       = base[d] + set bits of d's mask below i   (stable by construction)
+//   start of sub-bag (bag s, d) = base[d] + set bits of d's mask below the bag's first lookup
+// so neither needs a per-bag loop, an atomic or a second pass over the IDs, and the
+// sub-bag starts (bag-major [table][sample][dst]) are written with coalesced stores.
+#define BLS_RW_CHUNK (BLS_RW_PER_THREAD * BLS_ROUTE_TB)
+#define BLS_RW_WORDS (BLS_RW_CHUNK / 32)
+__global__ void __launch_bounds__(BLS_ROUTE_TB, 10) bls_rw_scatter_kernel(BlsParams p)
 {
-    __shared__ int cnt[BLS_MAX_RANKS][BLS_ROUTE_TB + 1];
-    __shared__ int s_local[BLS_RW_STAGE], s_out[BLS_RW_STAGE];
-    __shared__ unsigned char s_dst[BLS_RW_STAGE];
-    __shared__ int s_tcount[BLS_MAX_RANKS], s_toff[BLS_MAX_RANKS];
+    extern __shared__ unsigned rw_smem[];
+    // layout: mask[P][WORDS + 1] | id[CHUNK] | off[TB + 1] | base[P] | pre[P][WORDS + 2] (16-bit)
+    unsigned (*s_mask)[BLS_RW_WORDS + 1] = reinterpret_cast<unsigned (*)[BLS_RW_WORDS + 1]>(rw_smem);
+    int *s_id = reinterpret_cast<int *>(rw_smem + (size_t)p.P * (BLS_RW_WORDS + 1));
+    int *s_off = s_id + BLS_RW_CHUNK;
+    int *s_base = s_off + BLS_ROUTE_TB + 1;
+    unsigned short (*s_pre)[BLS_RW_WORDS + 2] = reinterpret_cast<unsigned short (*)[BLS_RW_WORDS + 2]>(s_base + p.P);
+
     const int src = blockIdx.y;
     RouteCtx c;
     if (!route_ctx(p, src, c)) return;
+    const int tid = threadIdx.x, lane = tid & 31, w = tid >> 5;
     const int t = blockIdx.x / p.tiles_per_table;
-    const int s0 = (blockIdx.x % p.tiles_per_table) * BLS_ROUTE_TB;
+    const int s0 = (blockIdx.x - t * p.tiles_per_table) * BLS_ROUTE_TB;
     const int nb = min(BLS_ROUTE_TB, p.b - s0);
-    const int s = threadIdx.x;
     const unsigned rows = (unsigned)p.tab[t].rows;
     const int blk = p.tab[t].blk;
     const unsigned magic = p.tab[t].magic;
     const long long g0 = ((long long)src * p.T + t) * p.b + s0;
-    for (int d = 0; d < p.P; d++) cnt[d][s] = 0;
     int lo, hi;
-    const bool ok = tile_range(p, c, g0, nb, lo, hi);
-    const bool staged = hi - lo <= BLS_RW_STAGE;
-    if (staged)
-        for (int l = lo + threadIdx.x; l < hi; l += BLS_ROUTE_TB) {
-            unsigned id = (unsigned)__ldcs(c.ids + l);
-            if (id >= rows) id = 0;
-            int local;
-            s_dst[l - lo] = (unsigned char)owner_of_row(id, blk, magic, local);
-            s_local[l - lo] = local;
-        }
-    __syncthreads();
-    int st = 0, en = 0;
-    if (ok && s < nb) { st = c.off[g0 + s]; en = c.off[g0 + s + 1]; }
-    auto look = [&](int l, int &local) {                    // owner and owner-local row of lookup l
-        if (staged) { local = s_local[l - lo]; return (int)s_dst[l - lo]; }
-        unsigned id = (unsigned)c.ids[l];
-        if (id >= rows) id = 0;
-        return owner_of_row(id, blk, magic, local);
-    };
-    for (int l = st; l < en; l++) { int local; cnt[look(l, local)][s]++; }
-    __syncthreads();
-    // exclusive scan over the bags of the tile, one warp per destination
-    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
-    const int *tb = p.tile_cnt + ((size_t)src * p.NT + blockIdx.x) * p.P;
-    for (int d = w; d < p.P; d += BLS_ROUTE_TB / 32) {
-        int v[BLS_ROUTE_TB / 32], tot = 0;
-        #pragma unroll
-        for (int q = 0; q < BLS_ROUTE_TB / 32; q++) { v[q] = cnt[d][lane * (BLS_ROUTE_TB / 32) + q]; tot += v[q]; }
-        int inc = tot;
-        for (int o = 1; o < 32; o <<= 1) {
-            int y = __shfl_up_sync(0xffffffffu, inc, o);
-            if (lane >= o) inc += y;
-        }
-        int run = tb[d] + inc - tot;
-        #pragma unroll
-        for (int q = 0; q < BLS_ROUTE_TB / 32; q++) { cnt[d][lane * (BLS_ROUTE_TB / 32) + q] = run; run += v[q]; }
-        if (lane == 31) s_tcount[d] = run - tb[d];          // lookups of this tile that go to d
+    tile_ends(p, c, g0, nb, lo, hi);
+    const int n = hi - lo;
+    // bag starts relative to the tile, forced into [0, n]; a bag that ends before it starts is reported
+    for (int s = tid; s <= nb; s += BLS_ROUTE_TB) {
+        const long long a = c.off[g0 + s];
+        if (s < nb && n > 0 && a > (long long)c.off[g0 + s + 1]) flag(p, BLS_ST_EINVAL);
+        s_off[s] = (int)min(max(a - lo, 0LL), (long long)n);
     }
-    __syncthreads();
-    // sub-bag starts of the tile: nb rows of P entries, contiguous in the bag-major layout
-    {
-        int *rows_out = c.sub_start + ((size_t)t * p.b + s0) * p.P;
-        for (int e = threadIdx.x; e < nb * p.P; e += BLS_ROUTE_TB) rows_out[e] = min(cnt[e % p.P][e / p.P], p.cap);
-    }
-    if (!staged) {                                          // oversized tile: write straight to the send buffer
-        for (int l = st; l < en; l++) {
+    if (tid < p.P) s_base[tid] = p.tile_cnt[((size_t)src * p.NT + blockIdx.x) * p.P + tid];
+    int *rows_out = c.sub_start + ((size_t)t * p.b + s0) * p.P;
+    const unsigned inv_p = (1u << 20) / (unsigned)p.P + 1u;     // e / P for e < 4096 as a multiply
+    const unsigned lt = (1u << lane) - 1u;
+
+    for (int c0 = 0; c0 == 0 || c0 < n; c0 += BLS_RW_CHUNK) {
+        const int nc = min(BLS_RW_CHUNK, n - c0);
+        const int nw = (nc + 31) >> 5;
+        const bool last = c0 + nc >= n;
+        // classify: all loads first (staged in shared memory, range-checked), then per warp
+        // step the lanes that share a destination find one another and one of them stores
+        // their mask; destinations nobody goes to keep the zero written just before
+        {
+            int idr[BLS_RW_PER_THREAD];
+            #pragma unroll
+            for (int q = 0; q < BLS_RW_PER_THREAD; q++) {
+                const int i = q * BLS_ROUTE_TB + tid;
+                idr[q] = i < nc ? __ldcs(c.ids + lo + c0 + i) : 0;
+            }
+            #pragma unroll
+            for (int q = 0; q < BLS_RW_PER_THREAD; q++) {
+                const int i = q * BLS_ROUTE_TB + tid;
+                if (i < nc) s_id[i] = (unsigned)idr[q] < rows ? idr[q] : 0;   // out of range: reported by the count kernel
+            }
+        }
+        #pragma unroll 1
+        for (int i = tid; i - lane < nc; i += BLS_ROUTE_TB) {           // the bound is the same for a whole warp
+            int d = 64 + lane;                                          // no lookup: matches nobody
+            if (i < nc) {
+                int local;
+                d = owner_of_row((unsigned)s_id[i], blk, magic, local);
+            }
+            if (lane < p.P) s_mask[lane][i >> 5] = 0u;
+            __syncwarp();
+            const unsigned same = __match_any_sync(0xffffffffu, d);
+            if (i < nc && lane == __ffs(same) - 1) s_mask[d][i >> 5] = same;
+        }
+        __syncthreads();
+        // set bits before every word, one warp per destination (two words per lane)
+        for (int d = w; d < p.P; d += BLS_ROUTE_TB / 32) {
+            const int v0 = 2 * lane < nw ? __popc(s_mask[d][2 * lane]) : 0;
+            const int v1 = 2 * lane + 1 < nw ? __popc(s_mask[d][2 * lane + 1]) : 0;
+            int inc = v0 + v1;
+            for (int o = 1; o < 32; o <<= 1) {
+                const int y = __shfl_up_sync(0xffffffffu, inc, o);
+                if (lane >= o) inc += y;
+            }
+            const int excl = inc - v0 - v1;
+            if (2 * lane < nw) s_pre[d][2 * lane] = (unsigned short)excl;
+            if (2 * lane + 1 < nw) s_pre[d][2 * lane + 1] = (unsigned short)(excl + v0);
+            if (lane == 31) { s_pre[d][nw] = (unsigned short)inc; s_mask[d][nw] = 0u; }   // closing entry: the chunk's total
+        }
+        __syncthreads();
+        for (int i = tid; i < nc; i += BLS_ROUTE_TB) {
             int local;
-            const int d = look(l, local);
-            const int pos = cnt[d][s]++;
+            const int d = owner_of_row((unsigned)s_id[i], blk, magic, local);
+            const int pos = s_base[d] + s_pre[d][i >> 5] + __popc(s_mask[d][i >> 5] & lt);
             if (pos < p.cap) c.sendbuf[pos] = local;
         }
-        return;
+        // bags that start inside this chunk (the last chunk also takes those that start at its end)
+        for (int e = tid; e < nb * p.P; e += BLS_ROUTE_TB) {
+            const int s = (int)(((unsigned)e * inv_p) >> 20);
+            const int d = e - s * p.P;
+            const int x = s_off[s] - c0;
+            if (x >= 0 && (x < nc || (last && x == nc))) {
+                const int v = s_base[d] + s_pre[d][x >> 5] + __popc(s_mask[d][x >> 5] & ((1u << (x & 31)) - 1u));
+                rows_out[e] = min(v, p.cap);
+            }
+        }
+        __syncthreads();
+        if (tid < p.P) s_base[tid] += s_pre[tid][nw];
+        __syncthreads();
     }
-    // reorder inside shared memory (destination-major, order kept), then copy each
-    // destination's segment to the send buffer with coalesced stores
-    if (threadIdx.x == 0) {
-        int run = 0;
-        for (int d = 0; d < p.P; d++) { s_toff[d] = run; run += s_tcount[d]; }
-    }
-    __syncthreads();
-    for (int l = st; l < en; l++) {
-        int local;
-        const int d = look(l, local);
-        const int pos = cnt[d][s]++;
-        s_out[s_toff[d] + (pos - tb[d])] = local;
-    }
-    __syncthreads();
-    for (int d = 0; d < p.P; d++) {
-        const int base_d = tb[d], n_d = s_tcount[d], o_d = s_toff[d];
-        for (int k2 = threadIdx.x; k2 < n_d; k2 += BLS_ROUTE_TB)
-            if (base_d + k2 < p.cap) c.sendbuf[base_d + k2] = s_out[o_d + k2];
-    }
+    // the entries after the last bag of the requester close every destination's region
+    if (blockIdx.x == p.NT - 1 && tid < p.P) c.sub_start[(size_t)p.T * p.b * p.P + tid] = min(s_base[tid], p.cap);
+}
+
+static size_t rw_scatter_smem(const BlsParams &p)
+{
+    return sizeof(unsigned) * (size_t)p.P * (BLS_RW_WORDS + 1) + sizeof(int) * (BLS_RW_CHUNK + BLS_ROUTE_TB + 1 + p.P) +
+           sizeof(unsigned short) * (size_t)p.P * (BLS_RW_WORDS + 2);
 }
 
 int bls_route_kernels(const bls_plan_t *pl) { return pl->prm.part == BLS_PART_TABLE_RR ? 1 : 3; }
@@ -315,6 +348,6 @@ void bls_launch_route(const bls_plan_t *pl)
     } else {
         bls_rw_count_kernel<<<grid, BLS_ROUTE_TB, 0, pl->stream>>>(p);
         bls_rw_scan_kernel<<<p.P, 1024, 0, pl->stream>>>(p);
-        bls_rw_scatter_kernel<<<grid, BLS_ROUTE_TB, 0, pl->stream>>>(p);
+        bls_rw_scatter_kernel<<<grid, BLS_ROUTE_TB, rw_scatter_smem(p), pl->stream>>>(p);
     }
 }
