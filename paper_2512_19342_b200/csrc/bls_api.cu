@@ -50,11 +50,11 @@ void fill_params(BlsParams &p, const bls_table_t *tables, int T, int part, int P
     p.cap = (int)((cap + 3) / 4 * 4);          // every rank's send buffer starts on a 16-byte boundary
     // Routing tiles.  Row-wise: BLS_ROUTE_TB bags (the scatter kernel's shared-memory tile).
     // Table-wise: a tile is only copied, so it grows for short bags until a block moves
-    // about 4096 IDs, as long as enough tiles remain to fill the GPU.
+    // 2048 IDs or more, as long as enough tiles remain to fill the GPU.
     p.tile_bags = BLS_ROUTE_TB;
     if (part == BLS_PART_TABLE_RR) {
         const double avg = (double)cap / ((double)p.NI * b);
-        while (p.tile_bags < b && p.tile_bags * avg < 4096.0 &&
+        while (p.tile_bags < b && p.tile_bags * avg < 2048.0 &&
                (long long)T * P * ((b + 2 * p.tile_bags - 1) / (2 * p.tile_bags)) >= 2048)
             p.tile_bags *= 2;
     }
@@ -238,6 +238,11 @@ void bls_destroy(bls_plan_t *plan)
         for (int i = 0; i < BLS_PROF_MAX * 4; i++) cudaEventDestroy(plan->prof_ev[i]);
         free(plan->prof_ev);
     }
+    if (plan->side_ready) {
+        cudaStreamDestroy(plan->s_side);
+        cudaEventDestroy(plan->e_fork);
+        cudaEventDestroy(plan->e_join);
+    }
     if (plan->host_path) {
         cudaStreamDestroy(plan->s_in);
         cudaStreamDestroy(plan->s_out);
@@ -252,6 +257,11 @@ void bls_destroy(bls_plan_t *plan)
 bls_status_t bls_profile(bls_plan_t *pl, int enable)
 {
     if (!pl) return BLS_EINVAL;
+    if (enable && !pl->prof_ev) {
+        pl->prof_ev = (cudaEvent_t *)calloc((size_t)BLS_PROF_MAX * 4, sizeof(cudaEvent_t));
+        if (!pl->prof_ev) return BLS_ENOSPC;
+        for (int i = 0; i < BLS_PROF_MAX * 4; i++) cudaEventCreate(&pl->prof_ev[i]);
+    }
     pl->prof_on = enable ? 1 : 0;
     return BLS_OK;
 }
@@ -290,14 +300,7 @@ static void enqueue_wave(bls_plan_t *pl, int mode, long long t_last, long long f
                          const int *ids, const int *off, long long n_ids, int opportunistic = 0)
 {
     cudaEvent_t *ev = nullptr;
-    if (pl->prof_on && pl->prof_n < BLS_PROF_MAX) {
-        if (!pl->prof_ev) {
-            pl->prof_ev = (cudaEvent_t *)calloc((size_t)BLS_PROF_MAX * 4, sizeof(cudaEvent_t));
-            if (pl->prof_ev)
-                for (int i = 0; i < BLS_PROF_MAX * 4; i++) cudaEventCreate(&pl->prof_ev[i]);
-        }
-        if (pl->prof_ev) ev = pl->prof_ev + (size_t)pl->prof_n++ * 4;
-    }
+    if (pl->prof_on && pl->prof_n < BLS_PROF_MAX && pl->prof_ev) ev = pl->prof_ev + (size_t)pl->prof_n++ * 4;
     if (ev) cudaEventRecord(ev[0], pl->stream);
     bls_launch_gate(pl, mode, t_last, floor_, k, ids, off, n_ids, opportunistic);
     bls_launch_route(pl);
@@ -305,6 +308,44 @@ static void enqueue_wave(bls_plan_t *pl, int mode, long long t_last, long long f
     bls_launch_gather(pl);                             // its last block commits the wave
     if (ev) { cudaEventRecord(ev[2], pl->stream); cudaEventRecord(ev[3], pl->stream); }
     pl->kernels_launched += 2 + bls_route_kernels(pl);
+}
+
+// Overlapped wave (bound >= 1): the requesters post iteration t while the owners answer
+// iteration t - 1, which is in another slot, so the two do not depend on each other
+// (Table I of the paper: communication of one batch beside computation of another).  The
+// gate plans both; then the gather kernel (answer t - 1, commit) goes to the plan's stream
+// and the router's copy kernel (post t) to a second stream, in blocks small enough to
+// fit beside the gather kernel's resident blocks.  The plan's stream waits for the copy
+// kernel, so everything enqueued on it afterwards sees the wave complete.
+static bool side_stream_ready(bls_plan_t *pl)
+{
+    if (pl->side_ready) return true;
+    if (cudaStreamCreateWithFlags(&pl->s_side, cudaStreamNonBlocking) != cudaSuccess) return false;
+    if (cudaEventCreateWithFlags(&pl->e_fork, cudaEventDisableTiming) != cudaSuccess ||
+        cudaEventCreateWithFlags(&pl->e_join, cudaEventDisableTiming) != cudaSuccess) {
+        cudaStreamDestroy(pl->s_side);
+        return false;
+    }
+    pl->side_ready = 1;
+    return true;
+}
+
+static void enqueue_wave_overlapped(bls_plan_t *pl, long long t_last, long long floor_, int k, const int *ids,
+                                    const int *off, long long n_ids)
+{
+    cudaEvent_t *ev = nullptr;
+    if (pl->prof_on && pl->prof_n < BLS_PROF_MAX && pl->prof_ev) ev = pl->prof_ev + (size_t)pl->prof_n++ * 4;
+    if (ev) cudaEventRecord(ev[0], pl->stream);
+    bls_launch_gate(pl, BLS_MODE_STEP, t_last, floor_, k, ids, off, n_ids, 0, 1);
+    cudaEventRecord(pl->e_fork, pl->stream);
+    if (ev) cudaEventRecord(ev[1], pl->stream);
+    bls_launch_gather(pl);                             // first, so that its blocks are resident first
+    cudaStreamWaitEvent(pl->s_side, pl->e_fork, 0);
+    bls_launch_route_beside(pl, pl->s_side);
+    cudaEventRecord(pl->e_join, pl->s_side);
+    cudaStreamWaitEvent(pl->stream, pl->e_join, 0);
+    if (ev) { cudaEventRecord(ev[2], pl->stream); cudaEventRecord(ev[3], pl->stream); }
+    pl->kernels_launched += 3;
 }
 
 // Debug aid: a slot that is about to receive iteration `iter` holds an iteration that has
@@ -362,9 +403,18 @@ bls_status_t bls_step(bls_plan_t *pl, int k, const int32_t *ids, const int32_t *
     // (while the iteration to hand back is incomplete they wait for the earliest rank that can act) let them drift apart and catch
     // up, the last wave enforces the bound.  Without delays one wave does everything.
     const int waves = pl->any_stall ? (pl->max_waves < pl->prm.P + 1 ? pl->max_waves : pl->prm.P + 1) : 1;
-    for (int v = 0; v + 1 < waves; v++)
-        enqueue_wave(pl, BLS_MODE_STEP, t, t - k, k, ids, v == 0 ? offsets : nullptr, n_ids, 1);
-    enqueue_wave(pl, BLS_MODE_STEP, t, t - k, k, ids, waves == 1 ? offsets : nullptr, n_ids);
+    // (iterations of a few thousand lookups are bound by the host's launch rate, and the
+    // second stream costs four more driver calls per step: they stay on one stream)
+    const bool overlapped = k >= 1 && !pl->any_stall && pl->prm.part == BLS_PART_TABLE_RR && !pl->prm.hot.enabled &&
+                            (long long)pl->prm.P * pl->prm.cap >= 16384 && side_stream_ready(pl);
+    if (overlapped) {
+        enqueue_wave_overlapped(pl, t, t - k, k, ids, offsets, n_ids);
+        pl->unserved = 1;                              // iteration t is answered by the next wave
+    } else {
+        for (int v = 0; v + 1 < waves; v++)
+            enqueue_wave(pl, BLS_MODE_STEP, t, t - k, k, ids, v == 0 ? offsets : nullptr, n_ids, 1);
+        enqueue_wave(pl, BLS_MODE_STEP, t, t - k, k, ids, waves == 1 ? offsets : nullptr, n_ids);
+    }
     if (t - k >= 0) {
         *out = slot_out(pl, t - k);
         *out_iter = t - k;
@@ -387,10 +437,13 @@ bls_status_t bls_drain(bls_plan_t *pl, const float **out, int64_t *out_iter)
         return BLS_OK;
     }
     const long long f = pl->t_handed;
-    // Without injected delays every rank completes an iteration in the step that
-    // issues it, so the outstanding iterations are already complete on the stream.
-    if (pl->any_stall)
+    // Without injected delays every rank completes an iteration in the step that issues
+    // it (in overlapped mode: in the step after it, so the newest one is still to be
+    // answered); otherwise the outstanding iterations are already complete on the stream.
+    if (pl->any_stall || pl->unserved) {
         enqueue_wave(pl, BLS_MODE_DRAIN, pl->t_next - 1, f, pl->k_cur < 0 ? 0 : pl->k_cur, nullptr, nullptr, 0);
+        pl->unserved = 0;
+    }
     *out = slot_out(pl, f);
     *out_iter = f;
     pl->t_handed = f + 1;

@@ -113,7 +113,8 @@ __device__ __forceinline__ void commit_lane(const BlsParams &p, int r)
             stall += z % (span + 1ull);
         }
         d->ready_ns[r] = now + stall;
-        d->route_iter[r] = -1;
+        // route_iter stays as it is until the next gate rewrites it: in overlapped mode the
+        // router of this wave may still be running beside the kernel that commits
     }
     j = d->serve_iter[r];
     if (j >= 0) {

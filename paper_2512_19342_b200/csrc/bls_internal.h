@@ -128,13 +128,20 @@ struct bls_plan {
     int max_waves;                // with injected delays: waves per step (the last one enforces the bound)
     int poison;                   // debug: fill an output slot with NaN patterns before an iteration is issued into it
     int hot_attached;             // a hot-row buffer has been attached
+    // overlapped mode (bound >= 1, table-wise, no injected delays): the router of iteration t
+    // runs on a stream of its own beside the gather kernel of iteration t - 1
+    cudaStream_t s_side;
+    cudaEvent_t e_fork, e_join;
+    int side_ready;
+    int unserved;                 // iterations posted whose answer has not been enqueued yet (0 or 1)
 };
 #define BLS_PROF_MAX 1024
 
 // kernel launchers (defined in the .cu files)
 void bls_launch_gate(const bls_plan_t *pl, int mode, long long t_last, long long forced_floor, int k,
-                     const int *ids, const int *off, long long n_ids, int opportunistic);
+                     const int *ids, const int *off, long long n_ids, int opportunistic, int overlapped = 0);
 void bls_launch_commit(const bls_plan_t *pl);
 void bls_launch_route(const bls_plan_t *pl);
+void bls_launch_route_beside(const bls_plan_t *pl, cudaStream_t stream);   // table-wise router sized to run beside the gather kernel
 void bls_launch_gather(const bls_plan_t *pl);
 int bls_route_kernels(const bls_plan_t *pl);   // kernels bls_launch_route enqueues

@@ -37,7 +37,8 @@ __device__ __forceinline__ long long warp_max_ll(long long v)
 // one more warp per rank, which then runs the first half of the router for the ranks
 // that were told to post (saves a launch on the critical path of every step).
 __device__ __forceinline__ void gate_warp(const BlsParams &p, int mode, long long t_last, long long floor_, int k,
-                                          const int *ids, const int *off, long long n_ids, int opportunistic)
+                                          const int *ids, const int *off, long long n_ids, int opportunistic,
+                                          int overlapped)
 {
     BlsDev *d = p.dev;
     const int r = threadIdx.x;
@@ -106,8 +107,11 @@ __device__ __forceinline__ void gate_warp(const BlsParams &p, int mode, long lon
     const long long min_posted2 = warp_min_ll(posted2);
     const long long max_posted2 = warp_max_ll(act ? posted2 : -1);
 
-    // serve: all P sources (self included) have posted the iteration
-    bool go_s = act && mode != BLS_MODE_ROUTE_ONLY && served < min_posted2 && is_ready;
+    // serve: all P sources (self included) have posted the iteration.  In overlapped mode the
+    // router of this wave runs beside the gather kernel, so only iterations posted by earlier
+    // waves can be answered.
+    const long long min_posted = warp_min_ll(posted);
+    bool go_s = act && mode != BLS_MODE_ROUTE_ONLY && served < (overlapped ? min_posted : min_posted2) && is_ready;
     if (p.part == BLS_PART_ROW_BLOCK) {
         // row-wise: a bag needs all owners' partial sums at once, so the owners answer an
         // iteration together, when all of them are free to act
@@ -139,9 +143,10 @@ __device__ __forceinline__ void gate_warp(const BlsParams &p, int mode, long lon
 
 __global__ void __launch_bounds__(1024) bls_gate_kernel(BlsParams p, int mode, long long t_last,
                                                         long long floor_, int k, const int *ids,
-                                                        const int *off, long long n_ids, int opportunistic)
+                                                        const int *off, long long n_ids, int opportunistic,
+                                                        int overlapped)
 {
-    if (threadIdx.x < 32) gate_warp(p, mode, t_last, floor_, k, ids, off, n_ids, opportunistic);
+    if (threadIdx.x < 32) gate_warp(p, mode, t_last, floor_, k, ids, off, n_ids, opportunistic, overlapped);
     if (p.part != BLS_PART_TABLE_RR || mode == BLS_MODE_LOOKUP_ONLY) return;
     __threadfence_block();
     __syncthreads();                                   // the wave plan is visible to the other warps
@@ -154,11 +159,11 @@ __global__ void __launch_bounds__(1024) bls_gate_kernel(BlsParams p, int mode, l
 __global__ void __launch_bounds__(32) bls_commit_kernel(BlsParams p) { commit_lane(p, threadIdx.x); }
 
 void bls_launch_gate(const bls_plan_t *pl, int mode, long long t_last, long long forced_floor, int k,
-                     const int *ids, const int *off, long long n_ids, int opportunistic)
+                     const int *ids, const int *off, long long n_ids, int opportunistic, int overlapped)
 {
     // table-wise: one warp per rank for the router's first half (warp 0 is also the gate)
     const bool meta = pl->prm.part == BLS_PART_TABLE_RR && mode != BLS_MODE_LOOKUP_ONLY;
-    bls_gate_kernel<<<1, meta ? 32 * pl->prm.P : 32, 0, pl->stream>>>(pl->prm, mode, t_last, forced_floor, k, ids, off, n_ids, opportunistic);
+    bls_gate_kernel<<<1, meta ? 32 * pl->prm.P : 32, 0, pl->stream>>>(pl->prm, mode, t_last, forced_floor, k, ids, off, n_ids, opportunistic, overlapped);
 }
 
 void bls_launch_commit(const bls_plan_t *pl)

@@ -22,7 +22,8 @@
 // bags, up to the whole chunk for short ones, so that a block always has a few
 // thousand IDs to move).  Copies the tile's IDs to their place in the send buffer
 // (coalesced) and writes the sub-bag starts.
-__global__ void __launch_bounds__(256) bls_tw_copy_kernel(BlsParams p)
+template <int INFLIGHT>
+__device__ __forceinline__ void tw_copy_tile(const BlsParams &p)
 {
     const int src = blockIdx.y;
     RouteCtx c;
@@ -50,15 +51,15 @@ __global__ void __launch_bounds__(256) bls_tw_copy_kernel(BlsParams p)
     const int lo = s_lo, hi = max(s_lo, s_hi);
     const int *in = c.ids + off0;
     if (!p.hot.enabled) {
-        for (int l0 = lo + threadIdx.x; l0 < hi; l0 += 4 * blockDim.x) {
-            int id[4];
+        for (int l0 = lo + threadIdx.x; l0 < hi; l0 += INFLIGHT * blockDim.x) {
+            int id[INFLIGHT];
             #pragma unroll
-            for (int q = 0; q < 4; q++) {
+            for (int q = 0; q < INFLIGHT; q++) {
                 const int l = l0 + q * blockDim.x;
                 id[q] = l < hi ? __ldcs(in + l) : 0;
             }
             #pragma unroll
-            for (int q = 0; q < 4; q++) {
+            for (int q = 0; q < INFLIGHT; q++) {
                 const int l = l0 + q * blockDim.x;
                 if (l >= hi) continue;
                 int v = id[q];
@@ -82,6 +83,13 @@ __global__ void __launch_bounds__(256) bls_tw_copy_kernel(BlsParams p)
         }
     }
 }
+
+__global__ void __launch_bounds__(256, 8) bls_tw_copy_kernel(BlsParams p) { tw_copy_tile<4>(p); }
+
+// The same router in blocks of 128 threads and at most 32 registers: one such block fits
+// on every SM beside the resident blocks of the gather kernel (3 x 256 threads x 80
+// registers), so that it can route the next iteration while the previous one is answered.
+__global__ void __launch_bounds__(128, 16) bls_tw_copy_beside_kernel(BlsParams p) { tw_copy_tile<8>(p); }
 
 // -------------------------------------------------------------------- row-wise
 
@@ -335,6 +343,12 @@ static size_t rw_scatter_smem(const BlsParams &p)
 {
     return sizeof(unsigned) * (size_t)p.P * (BLS_RW_WORDS + 1) + sizeof(int) * (BLS_RW_CHUNK + BLS_ROUTE_TB + 1 + p.P) +
            sizeof(unsigned short) * (size_t)p.P * (BLS_RW_WORDS + 2);
+}
+
+void bls_launch_route_beside(const bls_plan_t *pl, cudaStream_t stream)
+{
+    const BlsParams &p = pl->prm;
+    bls_tw_copy_beside_kernel<<<dim3(p.NT, p.P), 128, 0, stream>>>(p);
 }
 
 int bls_route_kernels(const bls_plan_t *pl) { return pl->prm.part == BLS_PART_TABLE_RR ? 1 : 3; }
