@@ -11,7 +11,7 @@ namespace {
 size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 struct Layout {
-    size_t dev, tab, pair, pair_of, pair_first, counts, sendbuf, sub_start, out, chunk_base, tile_cnt, stage_ids,
+    size_t dev, tab, pair, pair_of, pair_first, counts, sendbuf, sub_start, out, chunk_base, tile_cnt, rw_total, stage_ids,
         stage_off, total;
 };
 
@@ -82,6 +82,7 @@ Layout make_layout(const BlsParams &p)
     L.out = take(sizeof(float) * S * (size_t)p.out_slot_elems);
     L.chunk_base = take(sizeof(int) * P * (size_t)(p.NI + 1));
     L.tile_cnt = take(p.part == BLS_PART_ROW_BLOCK ? sizeof(int) * P * (size_t)p.NT * P : 0);
+    L.rw_total = take(p.part == BLS_PART_ROW_BLOCK ? sizeof(int) * P * P : 0);
     L.stage_ids = take(sizeof(int) * S * P * (size_t)p.cap);
     L.stage_off = take(sizeof(int) * S * ((size_t)P * p.T * p.b + 1));
     L.total = o;
@@ -147,6 +148,7 @@ bls_status_t bls_plan(const bls_table_t *tables, int T, int part, int P, int loc
     p.out = (float *)(ws + L.out);
     p.chunk_base = (int *)(ws + L.chunk_base);
     p.tile_cnt = (int *)(ws + L.tile_cnt);
+    p.rw_total = (int *)(ws + L.rw_total);
     p.stage_ids = (int *)(ws + L.stage_ids);
     p.stage_off = (int *)(ws + L.stage_off);
     pl->stream = (cudaStream_t)cuda_stream;
@@ -315,7 +317,9 @@ static void enqueue_wave(bls_plan_t *pl, int mode, long long t_last, long long f
 // (Table I of the paper: communication of one batch beside computation of another).  The
 // gate plans both; then the gather kernel (answer t - 1, commit) goes to the plan's stream
 // and the router's copy kernel (post t) to a second stream, in blocks small enough to
-// fit beside the gather kernel's resident blocks.  The plan's stream waits for the copy
+// fit beside the gather kernel's resident blocks.  (Row-wise placement stays sequential:
+// its router needs shared memory and several blocks per SM to hide its load latency,
+// neither of which the resident gather blocks leave.)  The plan's stream waits for the copy
 // kernel, so everything enqueued on it afterwards sees the wave complete.
 static bool side_stream_ready(bls_plan_t *pl)
 {
@@ -345,7 +349,7 @@ static void enqueue_wave_overlapped(bls_plan_t *pl, long long t_last, long long 
     cudaEventRecord(pl->e_join, pl->s_side);
     cudaStreamWaitEvent(pl->stream, pl->e_join, 0);
     if (ev) { cudaEventRecord(ev[2], pl->stream); cudaEventRecord(ev[3], pl->stream); }
-    pl->kernels_launched += 3;
+    pl->kernels_launched += 2 + bls_route_kernels(pl);
 }
 
 // Debug aid: a slot that is about to receive iteration `iter` holds an iteration that has

@@ -95,6 +95,7 @@ struct BlsParams {
     float *out;                  // [S][P][b][T][D]
     int *chunk_base;             // [P][NI+1]   table-wise: start of each (src, table) chunk
     int *tile_cnt;               // [P][NT][P]  row-wise: per tile, per destination counts / bases
+    int *rw_total;               // [P][P]      row-wise: lookups of requester src that go to d (zeroed by the gate)
     int *stage_ids;              // [S][P*cap]  staging for host inputs
     int *stage_off;              // [S][G+1]
     long long sub_stride;        // NQ + 1 rounded up to a multiple of 4

@@ -48,6 +48,8 @@ __device__ __forceinline__ void gate_warp(const BlsParams &p, int mode, long lon
     if (r == 0) { d->work_ctr = 0; d->done_ctr = 0; }
     if (p.hot.enabled)
         for (int i = r; i < p.NI; i += 32) p.hot.pair_ctr[i] = 0;
+    if (p.part == BLS_PART_ROW_BLOCK && mode != BLS_MODE_LOOKUP_ONLY)
+        for (int i = r; i < p.P * p.P; i += 32) p.rw_total[i] = 0;      // the count kernel adds the tiles' counts
     if (r == 0 && off != nullptr && (mode == BLS_MODE_STEP || mode == BLS_MODE_ROUTE_ONLY)) {
         int slot = (int)(t_last % p.S);
         d->in_ids[slot] = ids;

@@ -163,61 +163,70 @@ __global__ void __launch_bounds__(BLS_ROUTE_TB, 10) bls_rw_count_kernel(BlsParam
     }
     if (bad) flag(p, BLS_ST_ERANGE);
     __syncthreads();
-    if (tid < p.P) p.tile_cnt[((size_t)src * p.NT + blockIdx.x) * p.P + tid] = cnt[tid];
+    if (tid < p.P) {
+        p.tile_cnt[((size_t)src * p.NT + blockIdx.x) * p.P + tid] = cnt[tid];
+        if (cnt[tid]) atomicAdd(&p.rw_total[src * p.P + tid], cnt[tid]);
+    }
 }
 
-// One block per requester: exclusive scan of the tile counts in (destination, tile)
-// order, in place; send counts, displacements and the closing sub-bag entries.
-// Warp w owns destinations w, w+32, ...: totals first, then the displacements, then the
-// per-tile bases 32 tiles at a time.
-__global__ void __launch_bounds__(1024) bls_rw_scan_kernel(BlsParams p)
+// grid (P destinations, P requesters), 128 threads: displacement of the destination's
+// region (the totals of the destinations before it), send count, and the exclusive scan
+// of the destination's tile counts in tile order, in place.
+#define BLS_RW_SCAN_PER_THREAD 4
+__global__ void __launch_bounds__(128, 16) bls_rw_scan_kernel(BlsParams p)
 {
-    __shared__ long long tot[BLS_MAX_RANKS], disp[BLS_MAX_RANKS + 1];
-    const int src = blockIdx.x;
+    __shared__ long long s_disp;
+    __shared__ int s_warp[4];
+    const int d = blockIdx.x, src = blockIdx.y;
     RouteCtx c;
     if (!route_ctx(p, src, c)) return;
-    int *tc = p.tile_cnt + (size_t)src * p.NT * p.P;
-    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
-    for (int d = w; d < p.P; d += 32) {
-        long long sum = 0;
-        for (int tile = lane; tile < p.NT; tile += 32) sum += tc[(size_t)tile * p.P + d];
-        for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
-        if (lane == 0) tot[d] = sum;
-    }
-    __syncthreads();
-    if (threadIdx.x == 0) {
-        long long run = 0;
-        for (int d = 0; d < p.P; d++) { disp[d] = run; run += tot[d]; }
-        disp[p.P] = run;
-        if (run > p.cap) flag(p, BLS_ST_ENOSPC);
-    }
-    __syncthreads();
-    if (threadIdx.x < p.P) {
-        const int d = threadIdx.x;
-        c.sdispls[d] = (int)min(disp[d], (long long)0x7fffffff);
-        c.sendcounts[d] = (int)tot[d];
-    }
-    for (int d = w; d < p.P; d += 32) {
-        long long run = disp[d];
-        for (int t0 = 0; t0 < p.NT; t0 += 128) {           // four independent loads per lane in flight
-            int v[4];
-            #pragma unroll
-            for (int q = 0; q < 4; q++) {
-                const int tile = t0 + q * 32 + lane;
-                v[q] = tile < p.NT ? tc[(size_t)tile * p.P + d] : 0;
-            }
-            #pragma unroll
-            for (int q = 0; q < 4; q++) {
-                int inc = v[q];
-                for (int o = 1; o < 32; o <<= 1) {
-                    const int y = __shfl_up_sync(0xffffffffu, inc, o);
-                    if (lane >= o) inc += y;
-                }
-                const int tile = t0 + q * 32 + lane;
-                if (tile < p.NT) tc[(size_t)tile * p.P + d] = (int)min(run + inc - v[q], (long long)p.cap);
-                run += __shfl_sync(0xffffffffu, inc, 31);
-            }
+    const int tid = threadIdx.x, lane = tid & 31, w = tid >> 5;
+    if (w == 0) {
+        long long before = 0, all = 0;
+        for (int dd = lane; dd < p.P; dd += 32) {
+            const int x = p.rw_total[src * p.P + dd];
+            all += x;
+            if (dd < d) before += x;
         }
+        for (int o = 16; o > 0; o >>= 1) {
+            before += __shfl_xor_sync(0xffffffffu, before, o);
+            all += __shfl_xor_sync(0xffffffffu, all, o);
+        }
+        if (lane == 0) {
+            s_disp = before;
+            c.sdispls[d] = (int)min(before, (long long)0x7fffffff);
+            c.sendcounts[d] = p.rw_total[src * p.P + d];
+            if (d == 0 && all > p.cap) flag(p, BLS_ST_ENOSPC);
+        }
+    }
+    __syncthreads();
+    long long run = s_disp;
+    int *tc = p.tile_cnt + (size_t)src * p.NT * p.P + d;
+    for (int t0 = 0; t0 < p.NT; t0 += 128 * BLS_RW_SCAN_PER_THREAD) {
+        int v[BLS_RW_SCAN_PER_THREAD], sum = 0;
+        #pragma unroll
+        for (int q = 0; q < BLS_RW_SCAN_PER_THREAD; q++) {
+            const int tile = t0 + tid * BLS_RW_SCAN_PER_THREAD + q;
+            v[q] = tile < p.NT ? tc[(size_t)tile * p.P] : 0;
+            sum += v[q];
+        }
+        int inc = sum;
+        for (int o = 1; o < 32; o <<= 1) {
+            const int y = __shfl_up_sync(0xffffffffu, inc, o);
+            if (lane >= o) inc += y;
+        }
+        if (lane == 31) s_warp[w] = inc;
+        __syncthreads();
+        long long base = run + inc - sum;
+        for (int ww = 0; ww < w; ww++) base += s_warp[ww];
+        #pragma unroll
+        for (int q = 0; q < BLS_RW_SCAN_PER_THREAD; q++) {
+            const int tile = t0 + tid * BLS_RW_SCAN_PER_THREAD + q;
+            if (tile < p.NT) tc[(size_t)tile * p.P] = (int)min(base, (long long)p.cap);
+            base += v[q];
+        }
+        run += (long long)s_warp[0] + s_warp[1] + s_warp[2] + s_warp[3];
+        __syncthreads();
     }
 }
 
@@ -230,7 +239,7 @@ __global__ void __launch_bounds__(1024) bls_rw_scan_kernel(BlsParams p)
 //   start of sub-bag (bag s, d) = base[d] + set bits of d's mask below the bag's first lookup
 // so neither needs a per-bag loop, an atomic or a second pass over the IDs, and the
 // sub-bag starts (bag-major [table][sample][dst]) are written with coalesced stores.
-#define BLS_RW_CHUNK (BLS_RW_PER_THREAD * BLS_ROUTE_TB)
+#define BLS_RW_CHUNK 2048
 #define BLS_RW_WORDS (BLS_RW_CHUNK / 32)
 __global__ void __launch_bounds__(BLS_ROUTE_TB, 10) bls_rw_scatter_kernel(BlsParams p)
 {
@@ -274,16 +283,16 @@ __global__ void __launch_bounds__(BLS_ROUTE_TB, 10) bls_rw_scatter_kernel(BlsPar
         // classify: all loads first (staged in shared memory, range-checked), then per warp
         // step the lanes that share a destination find one another and one of them stores
         // their mask; destinations nobody goes to keep the zero written just before
-        {
+        for (int i0 = 0; i0 < nc; i0 += BLS_RW_PER_THREAD * BLS_ROUTE_TB) {
             int idr[BLS_RW_PER_THREAD];
             #pragma unroll
             for (int q = 0; q < BLS_RW_PER_THREAD; q++) {
-                const int i = q * BLS_ROUTE_TB + tid;
+                const int i = i0 + q * BLS_ROUTE_TB + tid;
                 idr[q] = i < nc ? __ldcs(c.ids + lo + c0 + i) : 0;
             }
             #pragma unroll
             for (int q = 0; q < BLS_RW_PER_THREAD; q++) {
-                const int i = q * BLS_ROUTE_TB + tid;
+                const int i = i0 + q * BLS_ROUTE_TB + tid;
                 if (i < nc) s_id[i] = (unsigned)idr[q] < rows ? idr[q] : 0;   // out of range: reported by the count kernel
             }
         }
@@ -361,7 +370,7 @@ void bls_launch_route(const bls_plan_t *pl)
         bls_tw_copy_kernel<<<grid, 256, 0, pl->stream>>>(p);
     } else {
         bls_rw_count_kernel<<<grid, BLS_ROUTE_TB, 0, pl->stream>>>(p);
-        bls_rw_scan_kernel<<<p.P, 1024, 0, pl->stream>>>(p);
+        bls_rw_scan_kernel<<<dim3(p.P, p.P), 128, 0, pl->stream>>>(p);
         bls_rw_scatter_kernel<<<grid, BLS_ROUTE_TB, rw_scatter_smem(p), pl->stream>>>(p);
     }
 }
