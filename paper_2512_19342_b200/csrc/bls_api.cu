@@ -48,10 +48,17 @@ void fill_params(BlsParams &p, const bls_table_t *tables, int T, int part, int P
     p.NI = part == BLS_PART_TABLE_RR ? T : T * P;
     p.NQ = p.NI * b;
     p.cap = (int)((cap + 3) / 4 * 4);          // every rank's send buffer starts on a 16-byte boundary
-    // Routing tiles.  Row-wise: BLS_ROUTE_TB bags (the scatter kernel's shared-memory tile).
+    // Routing tiles of BLS_ROUTE_TB bags or a power-of-two multiple.
     // Table-wise: a tile is only copied, so it grows for short bags until a block moves
     // 2048 IDs or more, as long as enough tiles remain to fill the GPU.
+    // Row-wise: up to 2048 bags (a tile is routed 2048 lookups at a time by one block, which
+    // requests the next 2048 while it works), fewer when the tiles would not fill the GPU.
     p.tile_bags = BLS_ROUTE_TB;
+    if (part == BLS_PART_ROW_BLOCK) {
+        while (p.tile_bags < b && p.tile_bags < 2048 &&
+               (long long)T * P * ((b + 2 * p.tile_bags - 1) / (2 * p.tile_bags)) >= 1024)
+            p.tile_bags *= 2;
+    }
     if (part == BLS_PART_TABLE_RR) {
         const double avg = (double)cap / ((double)p.NI * b);
         while (p.tile_bags < b && p.tile_bags * avg < 2048.0 &&

@@ -6,7 +6,7 @@
 
 #define BLS_MAX_RANKS 32
 #define BLS_MAX_SLOTS 16
-#define BLS_ROUTE_TB 128          // bags per routing tile (row-wise scatter: one thread per bag)
+#define BLS_ROUTE_TB 128          // smallest routing tile in bags; threads per block of the row-wise router
 
 // step modes understood by the gate kernel
 enum { BLS_MODE_STEP = 0, BLS_MODE_DRAIN = 1, BLS_MODE_ROUTE_ONLY = 2, BLS_MODE_LOOKUP_ONLY = 3 };
@@ -82,7 +82,7 @@ struct BlsParams {
     int cap;                // IDs per rank per iteration (send buffer capacity)
     int NT;                 // routing tiles per requester = T * tiles_per_table
     int tiles_per_table;    // ceil(b / tile_bags)
-    int tile_bags;          // bags per routing tile: BLS_ROUTE_TB row-wise, a multiple of it table-wise
+    int tile_bags;          // bags per routing tile: BLS_ROUTE_TB or a power-of-two multiple of it
     int row_bytes;
     BlsDev *dev;
     const BlsTableDesc *tab;     // [T]

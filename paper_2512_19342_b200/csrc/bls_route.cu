@@ -116,11 +116,14 @@ __device__ __forceinline__ void tile_ends(const BlsParams &p, const RouteCtx &c,
     lo = hi = 0;
 }
 
-// grid (NT, P), 128 threads: per-tile histogram over destinations.  All of a thread's
-// IDs are requested before the first one is used; lanes with the same destination are
-// counted together (one shared-memory atomic per distinct destination and warp step).
+// grid (NT, P), 128 threads: per-tile histogram over destinations (a tile is p.tile_bags
+// bags of one table of one requester, up to a whole chunk).  The tile's IDs are read 2048
+// at a time; the next 2048 are requested before the current ones are counted.  Lanes with
+// the same destination are counted together (one shared-memory atomic per distinct
+// destination and warp step).
 #define BLS_RW_PER_THREAD 16
-__global__ void __launch_bounds__(BLS_ROUTE_TB, 10) bls_rw_count_kernel(BlsParams p)
+#define BLS_RW_CHUNK (BLS_RW_PER_THREAD * BLS_ROUTE_TB)
+__global__ void __launch_bounds__(BLS_ROUTE_TB, 8) bls_rw_count_kernel(BlsParams p)
 {
     __shared__ int cnt[BLS_MAX_RANKS];
     const int src = blockIdx.y;
@@ -128,8 +131,8 @@ __global__ void __launch_bounds__(BLS_ROUTE_TB, 10) bls_rw_count_kernel(BlsParam
     if (!route_ctx(p, src, c)) return;
     const int tid = threadIdx.x, lane = tid & 31;
     const int t = blockIdx.x / p.tiles_per_table;
-    const int s0 = (blockIdx.x - t * p.tiles_per_table) * BLS_ROUTE_TB;
-    const int nb = min(BLS_ROUTE_TB, p.b - s0);
+    const int s0 = (blockIdx.x - t * p.tiles_per_table) * p.tile_bags;
+    const int nb = min(p.tile_bags, p.b - s0);
     if (tid < BLS_MAX_RANKS) cnt[tid] = 0;
     int lo, hi;
     tile_ends(p, c, ((long long)src * p.T + t) * p.b + s0, nb, lo, hi);
@@ -138,12 +141,17 @@ __global__ void __launch_bounds__(BLS_ROUTE_TB, 10) bls_rw_count_kernel(BlsParam
     const unsigned magic = p.tab[t].magic;
     __syncthreads();
     bool bad = false;
-    for (int l0 = lo; l0 < hi; l0 += BLS_RW_PER_THREAD * BLS_ROUTE_TB) {
-        int idr[BLS_RW_PER_THREAD];
+    int cur[BLS_RW_PER_THREAD], nxt[BLS_RW_PER_THREAD];
+    #pragma unroll
+    for (int q = 0; q < BLS_RW_PER_THREAD; q++) {
+        const int l = lo + q * BLS_ROUTE_TB + tid;
+        cur[q] = l < hi ? __ldcs(c.ids + l) : 0;
+    }
+    for (int l0 = lo; l0 < hi; l0 += BLS_RW_CHUNK) {
         #pragma unroll
         for (int q = 0; q < BLS_RW_PER_THREAD; q++) {
-            const int l = l0 + q * BLS_ROUTE_TB + tid;
-            idr[q] = l < hi ? __ldcs(c.ids + l) : 0;
+            const int l = l0 + BLS_RW_CHUNK + q * BLS_ROUTE_TB + tid;
+            nxt[q] = l < hi ? __ldcs(c.ids + l) : 0;
         }
         #pragma unroll
         for (int q = 0; q < BLS_RW_PER_THREAD; q++) {
@@ -151,7 +159,7 @@ __global__ void __launch_bounds__(BLS_ROUTE_TB, 10) bls_rw_count_kernel(BlsParam
             if (l - lane < hi) {                            // same for the whole warp
                 int d = 64 + lane;                          // no lookup: matches nobody
                 if (l < hi) {
-                    unsigned id = (unsigned)idr[q];
+                    unsigned id = (unsigned)cur[q];
                     if (id >= rows) { id = 0; bad = true; }
                     int local;
                     d = owner_of_row(id, blk, magic, local);
@@ -160,6 +168,8 @@ __global__ void __launch_bounds__(BLS_ROUTE_TB, 10) bls_rw_count_kernel(BlsParam
                 if (l < hi && lane == __ffs(same) - 1) atomicAdd(&cnt[d], __popc(same));
             }
         }
+        #pragma unroll
+        for (int q = 0; q < BLS_RW_PER_THREAD; q++) cur[q] = nxt[q];
     }
     if (bad) flag(p, BLS_ST_ERANGE);
     __syncthreads();
@@ -239,16 +249,15 @@ __global__ void __launch_bounds__(128, 16) bls_rw_scan_kernel(BlsParams p)
 //   start of sub-bag (bag s, d) = base[d] + set bits of d's mask below the bag's first lookup
 // so neither needs a per-bag loop, an atomic or a second pass over the IDs, and the
 // sub-bag starts (bag-major [table][sample][dst]) are written with coalesced stores.
-#define BLS_RW_CHUNK 2048
 #define BLS_RW_WORDS (BLS_RW_CHUNK / 32)
-__global__ void __launch_bounds__(BLS_ROUTE_TB, 10) bls_rw_scatter_kernel(BlsParams p)
+__global__ void __launch_bounds__(BLS_ROUTE_TB, 8) bls_rw_scatter_kernel(BlsParams p)
 {
     extern __shared__ unsigned rw_smem[];
-    // layout: mask[P][WORDS + 1] | id[CHUNK] | off[TB + 1] | base[P] | pre[P][WORDS + 2] (16-bit)
+    // layout: mask[P][WORDS + 1] | id[CHUNK] | off[tile_bags + 1] | base[P] | pre[P][WORDS + 2] (16-bit)
     unsigned (*s_mask)[BLS_RW_WORDS + 1] = reinterpret_cast<unsigned (*)[BLS_RW_WORDS + 1]>(rw_smem);
     int *s_id = reinterpret_cast<int *>(rw_smem + (size_t)p.P * (BLS_RW_WORDS + 1));
     int *s_off = s_id + BLS_RW_CHUNK;
-    int *s_base = s_off + BLS_ROUTE_TB + 1;
+    int *s_base = s_off + p.tile_bags + 1;
     unsigned short (*s_pre)[BLS_RW_WORDS + 2] = reinterpret_cast<unsigned short (*)[BLS_RW_WORDS + 2]>(s_base + p.P);
 
     const int src = blockIdx.y;
@@ -256,8 +265,8 @@ __global__ void __launch_bounds__(BLS_ROUTE_TB, 10) bls_rw_scatter_kernel(BlsPar
     if (!route_ctx(p, src, c)) return;
     const int tid = threadIdx.x, lane = tid & 31, w = tid >> 5;
     const int t = blockIdx.x / p.tiles_per_table;
-    const int s0 = (blockIdx.x - t * p.tiles_per_table) * BLS_ROUTE_TB;
-    const int nb = min(BLS_ROUTE_TB, p.b - s0);
+    const int s0 = (blockIdx.x - t * p.tiles_per_table) * p.tile_bags;
+    const int nb = min(p.tile_bags, p.b - s0);
     const unsigned rows = (unsigned)p.tab[t].rows;
     const int blk = p.tab[t].blk;
     const unsigned magic = p.tab[t].magic;
@@ -265,6 +274,16 @@ __global__ void __launch_bounds__(BLS_ROUTE_TB, 10) bls_rw_scatter_kernel(BlsPar
     int lo, hi;
     tile_ends(p, c, g0, nb, lo, hi);
     const int n = hi - lo;
+    // the IDs of a chunk are requested one chunk ahead and parked in registers
+    int idr[BLS_RW_PER_THREAD];
+    auto request = [&](int c0) {
+        #pragma unroll
+        for (int q = 0; q < BLS_RW_PER_THREAD; q++) {
+            const int i = c0 + q * BLS_ROUTE_TB + tid;
+            idr[q] = i < n ? __ldcs(c.ids + lo + i) : 0;
+        }
+    };
+    request(0);
     // bag starts relative to the tile, forced into [0, n]; a bag that ends before it starts is reported
     for (int s = tid; s <= nb; s += BLS_ROUTE_TB) {
         const long long a = c.off[g0 + s];
@@ -273,28 +292,33 @@ __global__ void __launch_bounds__(BLS_ROUTE_TB, 10) bls_rw_scatter_kernel(BlsPar
     }
     if (tid < p.P) s_base[tid] = p.tile_cnt[((size_t)src * p.NT + blockIdx.x) * p.P + tid];
     int *rows_out = c.sub_start + ((size_t)t * p.b + s0) * p.P;
-    const unsigned inv_p = (1u << 20) / (unsigned)p.P + 1u;     // e / P for e < 4096 as a multiply
     const unsigned lt = (1u << lane) - 1u;
+    int s_lo = 0;                                       // first bag that starts in the current chunk
 
     for (int c0 = 0; c0 == 0 || c0 < n; c0 += BLS_RW_CHUNK) {
         const int nc = min(BLS_RW_CHUNK, n - c0);
         const int nw = (nc + 31) >> 5;
         const bool last = c0 + nc >= n;
-        // classify: all loads first (staged in shared memory, range-checked), then per warp
-        // step the lanes that share a destination find one another and one of them stores
-        // their mask; destinations nobody goes to keep the zero written just before
-        for (int i0 = 0; i0 < nc; i0 += BLS_RW_PER_THREAD * BLS_ROUTE_TB) {
-            int idr[BLS_RW_PER_THREAD];
-            #pragma unroll
-            for (int q = 0; q < BLS_RW_PER_THREAD; q++) {
-                const int i = i0 + q * BLS_ROUTE_TB + tid;
-                idr[q] = i < nc ? __ldcs(c.ids + lo + c0 + i) : 0;
+        // classify: the chunk's IDs go to shared memory (range-checked), then per warp step
+        // the lanes that share a destination find one another and one of them stores their
+        // mask; destinations nobody goes to keep the zero written just before
+        #pragma unroll
+        for (int q = 0; q < BLS_RW_PER_THREAD; q++) {
+            const int i = q * BLS_ROUTE_TB + tid;
+            if (i < nc) s_id[i] = (unsigned)idr[q] < rows ? idr[q] : 0;   // out of range: reported by the count kernel
+        }
+        if (!last) request(c0 + BLS_RW_CHUNK);
+        __syncthreads();                                // also: s_off and s_base are in place
+        // bags that start in [c0, c0 + nc): the starts are sorted, so they are s_lo .. s_hi - 1
+        // (the last chunk also takes the bags that start at its end)
+        int s_hi = nb;
+        if (!last) {
+            int a = s_lo, e = nb;                       // first bag whose start is >= c0 + nc
+            while (a < e) {
+                const int m = (a + e) >> 1;
+                if (s_off[m] < c0 + nc) a = m + 1; else e = m;
             }
-            #pragma unroll
-            for (int q = 0; q < BLS_RW_PER_THREAD; q++) {
-                const int i = i0 + q * BLS_ROUTE_TB + tid;
-                if (i < nc) s_id[i] = (unsigned)idr[q] < rows ? idr[q] : 0;   // out of range: reported by the count kernel
-            }
+            s_hi = a;
         }
         #pragma unroll 1
         for (int i = tid; i - lane < nc; i += BLS_ROUTE_TB) {           // the bound is the same for a whole warp
@@ -330,16 +354,25 @@ __global__ void __launch_bounds__(BLS_ROUTE_TB, 10) bls_rw_scatter_kernel(BlsPar
             const int pos = s_base[d] + s_pre[d][i >> 5] + __popc(s_mask[d][i >> 5] & lt);
             if (pos < p.cap) c.sendbuf[pos] = local;
         }
-        // bags that start inside this chunk (the last chunk also takes those that start at its end)
-        for (int e = tid; e < nb * p.P; e += BLS_ROUTE_TB) {
-            const int s = (int)(((unsigned)e * inv_p) >> 20);
-            const int d = e - s * p.P;
-            const int x = s_off[s] - c0;
-            if (x >= 0 && (x < nc || (last && x == nc))) {
-                const int v = s_base[d] + s_pre[d][x >> 5] + __popc(s_mask[d][x >> 5] & ((1u << (x & 31)) - 1u));
-                rows_out[e] = min(v, p.cap);
+        // sub-bag starts of those bags: one thread per bag; the word and the bit mask of the
+        // rank query are the same for all destinations, and a bag's P entries are contiguous
+        // in the bag-major layout
+        for (int s = s_lo + tid; s < s_hi; s += BLS_ROUTE_TB) {
+            const int x = min(max(s_off[s] - c0, 0), nc);
+            const int wd = x >> 5;
+            const unsigned below = (1u << (x & 31)) - 1u;
+            auto start_of = [&](int d) {
+                return min(s_base[d] + (int)s_pre[d][wd] + __popc(s_mask[d][wd] & below), p.cap);
+            };
+            int *row = rows_out + (size_t)s * p.P;
+            if ((p.P & 3) == 0) {
+                for (int d = 0; d < p.P; d += 4)
+                    *reinterpret_cast<int4 *>(row + d) = make_int4(start_of(d), start_of(d + 1), start_of(d + 2), start_of(d + 3));
+            } else {
+                for (int d = 0; d < p.P; d++) row[d] = start_of(d);
             }
         }
+        s_lo = s_hi;
         __syncthreads();
         if (tid < p.P) s_base[tid] += s_pre[tid][nw];
         __syncthreads();
@@ -350,7 +383,7 @@ __global__ void __launch_bounds__(BLS_ROUTE_TB, 10) bls_rw_scatter_kernel(BlsPar
 
 static size_t rw_scatter_smem(const BlsParams &p)
 {
-    return sizeof(unsigned) * (size_t)p.P * (BLS_RW_WORDS + 1) + sizeof(int) * (BLS_RW_CHUNK + BLS_ROUTE_TB + 1 + p.P) +
+    return sizeof(unsigned) * (size_t)p.P * (BLS_RW_WORDS + 1) + sizeof(int) * (BLS_RW_CHUNK + p.tile_bags + 1 + p.P) +
            sizeof(unsigned short) * (size_t)p.P * (BLS_RW_WORDS + 2);
 }
 

@@ -104,6 +104,8 @@ CASES = [
                                                       partition="row_block", lengths="extremes")),
     ("long_bags_rowwise", lambda: bi.tiny_workload(T=2, P=3, b=130, rows=900, dim=16, partition="row_block",
                                                    lengths="extremes")),    # two tiles per table, thousands of lookups per tile
+    ("rowwise_wide_tiles", lambda: bi.tiny_workload(T=8, P=8, b=4096, rows=5000, dim=8, partition="row_block",
+                                                    lengths="poisson10")),   # tiles of 256 bags, routed in two passes each
     ("short_bags_wide_tiles", lambda: bi.tiny_workload(T=9, P=4, b=700, rows=50, dim=8, lengths="pareto15c")),  # table-wise tiles of 256+ bags
     ("many_tables", lambda: bi.tiny_workload(T=70, P=3, b=9, rows=40, dim=16, lengths="mixed")),           # > 32 (owner, table) pairs
     ("max_ranks", lambda: bi.tiny_workload(T=40, P=32, b=5, rows=64, dim=32, lengths="poisson10")),
