@@ -84,12 +84,10 @@ __device__ __forceinline__ void tw_copy_tile(const BlsParams &p)
     }
 }
 
-__global__ void __launch_bounds__(256, 8) bls_tw_copy_kernel(BlsParams p) { tw_copy_tile<4>(p); }
-
-// The same router in blocks of 128 threads and at most 32 registers: one such block fits
-// on every SM beside the resident blocks of the gather kernel (3 x 256 threads x 80
-// registers), so that it can route the next iteration while the previous one is answered.
-__global__ void __launch_bounds__(128, 16) bls_tw_copy_beside_kernel(BlsParams p) { tw_copy_tile<8>(p); }
+// Blocks of 128 threads and at most 32 registers: one such block fits on every SM beside
+// the resident blocks of the gather kernel (3 x 256 threads x 80 registers), so that the
+// router can work on the next iteration while the previous one is answered.
+__global__ void __launch_bounds__(128, 16) bls_tw_copy_kernel(BlsParams p) { tw_copy_tile<8>(p); }
 
 // -------------------------------------------------------------------- row-wise
 
@@ -390,7 +388,7 @@ static size_t rw_scatter_smem(const BlsParams &p)
 void bls_launch_route_beside(const bls_plan_t *pl, cudaStream_t stream)
 {
     const BlsParams &p = pl->prm;
-    bls_tw_copy_beside_kernel<<<dim3(p.NT, p.P), 128, 0, stream>>>(p);
+    bls_tw_copy_kernel<<<dim3(p.NT, p.P), 128, 0, stream>>>(p);
 }
 
 int bls_route_kernels(const bls_plan_t *pl) { return pl->prm.part == BLS_PART_TABLE_RR ? 1 : 3; }
@@ -400,7 +398,7 @@ void bls_launch_route(const bls_plan_t *pl)
     const BlsParams &p = pl->prm;
     dim3 grid(p.NT, p.P);
     if (p.part == BLS_PART_TABLE_RR) {
-        bls_tw_copy_kernel<<<grid, 256, 0, pl->stream>>>(p);
+        bls_tw_copy_kernel<<<grid, 128, 0, pl->stream>>>(p);
     } else {
         bls_rw_count_kernel<<<grid, BLS_ROUTE_TB, 0, pl->stream>>>(p);
         bls_rw_scan_kernel<<<dim3(p.P, p.P), 128, 0, pl->stream>>>(p);
