@@ -70,7 +70,9 @@ typedef struct {
 /* Device pointers to the routing artefacts and output of one iteration's slot
  * (for parity checks and for consumers of the output).
  *   sendcounts/sdispls  [P][P] indexed [src][dst]   (alltoallv arguments of the request leg)
- *   recvcounts/rdispls  [P][P] indexed [dst][src]   (valid once the iteration has been looked up)
+ *   recvcounts/rdispls  [P][P] indexed [dst][src]   (valid once the owners have answered the iteration:
+ *                       bls_counters reports served > iter; with a bound >= 1 that may be one
+ *                       step after the step that issued it)
  *   sendbuf             rank src's packed send buffer starts at sendbuf + src*sendbuf_stride;
  *                       owner-local rows, sorted by dst, ties in original order
  *   sub_start           rank src's array starts at sub_start + src*sub_stride and has sub_entries
@@ -133,6 +135,16 @@ bls_status_t bls_lookup(bls_plan_t *plan, int64_t iter);
  *           while t < k.  `*out` stays valid until the next bls_step/bls_drain
  *           call on the stream.  ids/offsets of iteration t are borrowed until
  *           k further steps (or the drain) have run.
+ *           With k >= 1, table-wise placement, no injected delays and iterations of
+ *           more than a few thousand lookups, a step works in overlapped mode (the
+ *           paper's Table I: communication of one batch beside computation of another):
+ *           the requesters post iteration t while the owners answer iteration t-1, the
+ *           router running on a second stream beside the gather-pool kernel.  The
+ *           plan's stream waits for that second stream before the call returns control of
+ *           it, so the caller sees one ordered stream.  In this mode the owners are one
+ *           iteration behind the requesters after a step (bls_status reports a lag of 1)
+ *           and the first bls_drain call enqueues the last answer.  Results are the same
+ *           bit for bit in both modes.
  * bls_drain: Listing 2's final loop, one outstanding iteration per call, oldest
  *           first; *out = NULL once nothing is outstanding. */
 bls_status_t bls_step(bls_plan_t *plan, int k, const int32_t *ids, const int32_t *offsets,
