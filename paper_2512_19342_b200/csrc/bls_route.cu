@@ -250,13 +250,12 @@ __global__ void __launch_bounds__(128, 16) bls_rw_scan_kernel(BlsParams p)
 #define BLS_RW_WORDS (BLS_RW_CHUNK / 32)
 __global__ void __launch_bounds__(BLS_ROUTE_TB, 8) bls_rw_scatter_kernel(BlsParams p)
 {
-    extern __shared__ unsigned rw_smem[];
-    // layout: mask[P][WORDS + 1] | id[CHUNK] | off[tile_bags + 1] | base[P] | pre[P][WORDS + 2] (16-bit)
-    unsigned (*s_mask)[BLS_RW_WORDS + 1] = reinterpret_cast<unsigned (*)[BLS_RW_WORDS + 1]>(rw_smem);
-    int *s_id = reinterpret_cast<int *>(rw_smem + (size_t)p.P * (BLS_RW_WORDS + 1));
+    extern __shared__ __align__(8) unsigned rw_smem[];
+    // layout: mp[P][WORDS + 1] (x = mask word, y = set bits before it) | id[CHUNK] | off[tile_bags + 1] | base[P]
+    uint2 (*s_mp)[BLS_RW_WORDS + 1] = reinterpret_cast<uint2 (*)[BLS_RW_WORDS + 1]>(rw_smem);
+    int *s_id = reinterpret_cast<int *>(rw_smem + 2 * (size_t)p.P * (BLS_RW_WORDS + 1));
     int *s_off = s_id + BLS_RW_CHUNK;
     int *s_base = s_off + p.tile_bags + 1;
-    unsigned short (*s_pre)[BLS_RW_WORDS + 2] = reinterpret_cast<unsigned short (*)[BLS_RW_WORDS + 2]>(s_base + p.P);
 
     const int src = blockIdx.y;
     RouteCtx c;
@@ -325,31 +324,32 @@ __global__ void __launch_bounds__(BLS_ROUTE_TB, 8) bls_rw_scatter_kernel(BlsPara
                 int local;
                 d = owner_of_row((unsigned)s_id[i], blk, magic, local);
             }
-            if (lane < p.P) s_mask[lane][i >> 5] = 0u;
+            if (lane < p.P) s_mp[lane][i >> 5].x = 0u;
             __syncwarp();
             const unsigned same = __match_any_sync(0xffffffffu, d);
-            if (i < nc && lane == __ffs(same) - 1) s_mask[d][i >> 5] = same;
+            if (i < nc && lane == __ffs(same) - 1) s_mp[d][i >> 5].x = same;
         }
         __syncthreads();
         // set bits before every word, one warp per destination (two words per lane)
         for (int d = w; d < p.P; d += BLS_ROUTE_TB / 32) {
-            const int v0 = 2 * lane < nw ? __popc(s_mask[d][2 * lane]) : 0;
-            const int v1 = 2 * lane + 1 < nw ? __popc(s_mask[d][2 * lane + 1]) : 0;
+            const int v0 = 2 * lane < nw ? __popc(s_mp[d][2 * lane].x) : 0;
+            const int v1 = 2 * lane + 1 < nw ? __popc(s_mp[d][2 * lane + 1].x) : 0;
             int inc = v0 + v1;
             for (int o = 1; o < 32; o <<= 1) {
                 const int y = __shfl_up_sync(0xffffffffu, inc, o);
                 if (lane >= o) inc += y;
             }
             const int excl = inc - v0 - v1;
-            if (2 * lane < nw) s_pre[d][2 * lane] = (unsigned short)excl;
-            if (2 * lane + 1 < nw) s_pre[d][2 * lane + 1] = (unsigned short)(excl + v0);
-            if (lane == 31) { s_pre[d][nw] = (unsigned short)inc; s_mask[d][nw] = 0u; }   // closing entry: the chunk's total
+            if (2 * lane < nw) s_mp[d][2 * lane].y = (unsigned)excl;
+            if (2 * lane + 1 < nw) s_mp[d][2 * lane + 1].y = (unsigned)(excl + v0);
+            if (lane == 31) s_mp[d][nw] = make_uint2(0u, (unsigned)inc);   // closing entry: the chunk's total
         }
         __syncthreads();
         for (int i = tid; i < nc; i += BLS_ROUTE_TB) {
             int local;
             const int d = owner_of_row((unsigned)s_id[i], blk, magic, local);
-            const int pos = s_base[d] + s_pre[d][i >> 5] + __popc(s_mask[d][i >> 5] & lt);
+            const uint2 mp = s_mp[d][i >> 5];
+            const int pos = s_base[d] + (int)mp.y + __popc(mp.x & lt);
             if (pos < p.cap) c.sendbuf[pos] = local;
         }
         // sub-bag starts of those bags: one thread per bag; the word and the bit mask of the
@@ -360,7 +360,8 @@ __global__ void __launch_bounds__(BLS_ROUTE_TB, 8) bls_rw_scatter_kernel(BlsPara
             const int wd = x >> 5;
             const unsigned below = (1u << (x & 31)) - 1u;
             auto start_of = [&](int d) {
-                return min(s_base[d] + (int)s_pre[d][wd] + __popc(s_mask[d][wd] & below), p.cap);
+                const uint2 mp = s_mp[d][wd];
+                return min(s_base[d] + (int)mp.y + __popc(mp.x & below), p.cap);
             };
             int *row = rows_out + (size_t)s * p.P;
             if ((p.P & 3) == 0) {
@@ -372,7 +373,7 @@ __global__ void __launch_bounds__(BLS_ROUTE_TB, 8) bls_rw_scatter_kernel(BlsPara
         }
         s_lo = s_hi;
         __syncthreads();
-        if (tid < p.P) s_base[tid] += s_pre[tid][nw];
+        if (tid < p.P) s_base[tid] += (int)s_mp[tid][nw].y;
         __syncthreads();
     }
     // the entries after the last bag of the requester close every destination's region
@@ -381,8 +382,7 @@ __global__ void __launch_bounds__(BLS_ROUTE_TB, 8) bls_rw_scatter_kernel(BlsPara
 
 static size_t rw_scatter_smem(const BlsParams &p)
 {
-    return sizeof(unsigned) * (size_t)p.P * (BLS_RW_WORDS + 1) + sizeof(int) * (BLS_RW_CHUNK + p.tile_bags + 1 + p.P) +
-           sizeof(unsigned short) * (size_t)p.P * (BLS_RW_WORDS + 2);
+    return sizeof(uint2) * (size_t)p.P * (BLS_RW_WORDS + 1) + sizeof(int) * (BLS_RW_CHUNK + p.tile_bags + 1 + p.P);
 }
 
 void bls_launch_route_beside(const bls_plan_t *pl, cudaStream_t stream)

@@ -132,6 +132,39 @@ def test_bound_of_one_or_more_routes_beside_the_previous_answer():
     assert bls.bls_status(plan) == (bls.BLS_OK, 1)
 
 
+def test_delays_switched_on_and_off_mid_flight():
+    """A loop that starts in overlapped mode (bound 2, no delays), gets a delayed rank after
+    three steps (from then on the plan works in waves on one stream) and loses the delay again
+    after six: the owners' one-iteration backlog is carried over, every iteration comes back
+    once, in order, unchanged."""
+    w = bi.workload(2, 0.05, 0.25)
+    tabs = dev_tables(w, [bi.table_values(t) for t in w.tables])
+    n_iter = 9
+    ref, inputs, *_ = run_loop(w, tabs, 0, n_iter)
+    plan = make_plan(w, tabs, 2)
+    got = []
+    for t, (ids, off) in enumerate(inputs):
+        if t == 3:
+            bls.bls_set_stall(plan, 1, 400_000)
+        if t == 6:
+            bls.bls_set_stall(plan, 1, 0)
+        out, it = bls.bls_step(plan, 2, torch.from_numpy(ids).cuda(), torch.from_numpy(off).cuda())
+        if out is not None:
+            assert it == len(got)
+            got.append(out.clone())
+    while True:
+        out, it = bls.bls_drain(plan)
+        if out is None:
+            break
+        assert it == len(got)
+        got.append(out.clone())
+    status, lag = bls.bls_status(plan)
+    assert status == bls.BLS_OK and lag <= 2 and len(got) == n_iter
+    assert all(torch.equal(got[i], ref[i]) for i in range(n_iter))
+    posted, served, done = bls.bls_counters(plan)
+    assert posted == served == done == [n_iter] * w.P
+
+
 def test_changing_k_mid_flight_is_refused():
     w = bi.workload(1)
     tabs = dev_tables(w, [bi.table_values(t) for t in w.tables])
