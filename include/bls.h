@@ -135,8 +135,8 @@ bls_status_t bls_lookup(bls_plan_t *plan, int64_t iter);
  *           while t < k.  `*out` stays valid until the next bls_step/bls_drain
  *           call on the stream.  ids/offsets of iteration t are borrowed until
  *           k further steps (or the drain) have run.
- *           With k >= 1, table-wise placement, no injected delays and iterations of
- *           more than a few thousand lookups, a step works in overlapped mode (the
+ *           With k >= 1, table-wise placement, no injected delays and iterations of about
+ *           a million lookups or more (bls_set_overlap), a step works in overlapped mode (the
  *           paper's Table I: communication of one batch beside computation of another):
  *           the requesters post iteration t while the owners answer iteration t-1, the
  *           router running on a second stream beside the gather-pool kernel.  The
@@ -185,6 +185,11 @@ bls_status_t bls_set_random_stall(bls_plan_t *plan, int rank, int64_t max_ns, ui
  * earliest rank that can act (not for all of them), so ranks act at different moments and
  * faster ones run ahead; once it is complete waves do not wait; the last wave enforces the bound. */
 bls_status_t bls_set_waves_per_step(bls_plan_t *plan, int waves);
+/* Overlapped mode of bls_step (see there): mode 0 (default) uses it for iterations of about a
+ * million lookups or more (P * max_ids_per_rank >= 2^20; smaller ones are bound by the launch
+ * rate and lose to the second stream's extra driver calls), 1 whenever it applies (bound >= 1,
+ * table-wise placement, no injected delays, no hot-row staging), -1 never.  May be called at any time. */
+bls_status_t bls_set_overlap(bls_plan_t *plan, int mode);
 /* Debug aid: while enabled, the output slot an iteration is issued into is first filled
  * with 0xFF bytes (NaN), so that a bag that was not written, or a slot read before its data
  * arrived, shows up in the result.  Costs one pass over the slot per step. */

@@ -25,7 +25,7 @@ EXPORTS = ["bls_plan_bytes", "bls_plan", "bls_destroy", "bls_route", "bls_lookup
            "bls_drain", "bls_step_host", "bls_drain_host", "bls_view", "bls_counters", "bls_status",
            "bls_set_stall", "bls_set_wait_limit", "bls_strerror", "bls_fill_hash_table",
            "bls_profile", "bls_profile_read", "bls_set_tuning", "bls_route_table_rr_static",
-           "bls_set_random_stall", "bls_set_waves_per_step", "bls_set_poison", "bls_a2a_bytes", "bls_a2a_create", "bls_a2a_destroy", "bls_a2a_post", "bls_a2a_wait",
+           "bls_set_random_stall", "bls_set_waves_per_step", "bls_set_poison", "bls_set_overlap", "bls_a2a_bytes", "bls_a2a_create", "bls_a2a_destroy", "bls_a2a_post", "bls_a2a_wait",
            "bls_a2a_status", "bls_hot_bytes", "bls_hot_attach", "bls_hot_observe", "bls_hot_build", "bls_hot_view"]
 
 
@@ -219,6 +219,11 @@ def bls_set_waves_per_step(plan: Plan, waves: int) -> None:
 
 def bls_set_poison(plan: Plan, enable: bool) -> None:
     _check(lib().bls_set_poison(plan.handle, int(enable)), "bls_set_poison")
+
+
+def bls_set_overlap(plan: Plan, mode: int) -> None:
+    """-1 never, 0 by iteration size (default), 1 whenever the overlapped mode applies."""
+    _check(lib().bls_set_overlap(plan.handle, int(mode)), "bls_set_overlap")
 
 
 def bls_set_wait_limit(plan: Plan, ns: int) -> None:

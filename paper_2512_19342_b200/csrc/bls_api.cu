@@ -323,8 +323,8 @@ static void enqueue_wave(bls_plan_t *pl, int mode, long long t_last, long long f
 // iteration t - 1, which is in another slot, so the two do not depend on each other
 // (Table I of the paper: communication of one batch beside computation of another).  The
 // gate plans both; then the gather kernel (answer t - 1, commit) goes to the plan's stream
-// and the router's copy kernel (post t) to a second stream, in blocks small enough to
-// fit beside the gather kernel's resident blocks.  (Row-wise placement stays sequential:
+// and the router's two kernels (post t) to a second stream, the copy kernel in blocks small
+// enough to fit beside the gather kernel's resident blocks.  (Row-wise placement stays sequential:
 // its router needs shared memory and several blocks per SM to hide its load latency,
 // neither of which the resident gather blocks leave.)  The plan's stream waits for the copy
 // kernel, so everything enqueued on it afterwards sees the wave complete.
@@ -352,11 +352,12 @@ static void enqueue_wave_overlapped(bls_plan_t *pl, long long t_last, long long 
     if (ev) cudaEventRecord(ev[1], pl->stream);
     bls_launch_gather(pl);                             // first, so that its blocks are resident first
     cudaStreamWaitEvent(pl->s_side, pl->e_fork, 0);
+    bls_launch_meta(pl, pl->s_side);                   // chunk bases, send counts and displacements of iteration t
     bls_launch_route_beside(pl, pl->s_side);
     cudaEventRecord(pl->e_join, pl->s_side);
     cudaStreamWaitEvent(pl->stream, pl->e_join, 0);
     if (ev) { cudaEventRecord(ev[2], pl->stream); cudaEventRecord(ev[3], pl->stream); }
-    pl->kernels_launched += 2 + bls_route_kernels(pl);
+    pl->kernels_launched += 3 + bls_route_kernels(pl);
 }
 
 // Debug aid: a slot that is about to receive iteration `iter` holds an iteration that has
@@ -414,10 +415,11 @@ bls_status_t bls_step(bls_plan_t *pl, int k, const int32_t *ids, const int32_t *
     // (while the iteration to hand back is incomplete they wait for the earliest rank that can act) let them drift apart and catch
     // up, the last wave enforces the bound.  Without delays one wave does everything.
     const int waves = pl->any_stall ? (pl->max_waves < pl->prm.P + 1 ? pl->max_waves : pl->prm.P + 1) : 1;
-    // (iterations of a few thousand lookups are bound by the host's launch rate, and the
-    // second stream costs four more driver calls per step: they stay on one stream)
+    // (iterations below about a million lookups are bound by the launch rate, of the host or of
+    // the GPU, and the second stream costs five more driver calls per step: they stay on one stream)
     const bool overlapped = k >= 1 && !pl->any_stall && pl->prm.part == BLS_PART_TABLE_RR && !pl->prm.hot.enabled &&
-                            (long long)pl->prm.P * pl->prm.cap >= 16384 && side_stream_ready(pl);
+                            pl->overlap_mode >= 0 &&
+                            (pl->overlap_mode > 0 || (long long)pl->prm.P * pl->prm.cap >= (1 << 20)) && side_stream_ready(pl);
     if (overlapped) {
         enqueue_wave_overlapped(pl, t, t - k, k, ids, offsets, n_ids);
         pl->unserved = 1;                              // iteration t is answered by the next wave
@@ -612,6 +614,13 @@ bls_status_t bls_set_poison(bls_plan_t *pl, int enable)
 {
     if (!pl) return BLS_EINVAL;
     pl->poison = enable ? 1 : 0;
+    return BLS_OK;
+}
+
+bls_status_t bls_set_overlap(bls_plan_t *pl, int mode)
+{
+    if (!pl || mode < -1 || mode > 1) return BLS_EINVAL;
+    pl->overlap_mode = mode;
     return BLS_OK;
 }
 

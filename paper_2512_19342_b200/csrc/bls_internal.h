@@ -135,6 +135,7 @@ struct bls_plan {
     cudaEvent_t e_fork, e_join;
     int side_ready;
     int unserved;                 // iterations posted whose answer has not been enqueued yet (0 or 1)
+    int overlap_mode;             // -1 never, 0 chosen by the size of an iteration, 1 whenever the mode applies
 };
 #define BLS_PROF_MAX 1024
 
@@ -142,6 +143,7 @@ struct bls_plan {
 void bls_launch_gate(const bls_plan_t *pl, int mode, long long t_last, long long forced_floor, int k,
                      const int *ids, const int *off, long long n_ids, int opportunistic, int overlapped = 0);
 void bls_launch_commit(const bls_plan_t *pl);
+void bls_launch_meta(const bls_plan_t *pl, cudaStream_t stream);   // table-wise router, first half, as a kernel of its own
 void bls_launch_route(const bls_plan_t *pl);
 void bls_launch_route_beside(const bls_plan_t *pl, cudaStream_t stream);   // table-wise router sized to run beside the gather kernel
 void bls_launch_gather(const bls_plan_t *pl);

@@ -149,11 +149,24 @@ __global__ void __launch_bounds__(1024) bls_gate_kernel(BlsParams p, int mode, l
                                                         int overlapped)
 {
     if (threadIdx.x < 32) gate_warp(p, mode, t_last, floor_, k, ids, off, n_ids, opportunistic, overlapped);
-    if (p.part != BLS_PART_TABLE_RR || mode == BLS_MODE_LOOKUP_ONLY) return;
+    // overlapped mode: the router's first half runs on the second stream too (bls_tw_meta_kernel)
+    if (p.part != BLS_PART_TABLE_RR || mode == BLS_MODE_LOOKUP_ONLY || overlapped) return;
     __threadfence_block();
     __syncthreads();                                   // the wave plan is visible to the other warps
     const int w = threadIdx.x >> 5;
     if (w < p.P) tw_meta_warp(p, w, threadIdx.x & 31);
+}
+
+// The router's first half on its own (one warp per requester), for the overlapped mode.
+__global__ void __launch_bounds__(1024) bls_tw_meta_kernel(BlsParams p)
+{
+    const int w = threadIdx.x >> 5;
+    if (w < p.P) tw_meta_warp(p, w, threadIdx.x & 31);
+}
+
+void bls_launch_meta(const bls_plan_t *pl, cudaStream_t stream)
+{
+    bls_tw_meta_kernel<<<1, 32 * pl->prm.P, 0, stream>>>(pl->prm);
 }
 
 // One warp; publishes the progress of a wave that has no gather kernel at its end
@@ -164,7 +177,7 @@ void bls_launch_gate(const bls_plan_t *pl, int mode, long long t_last, long long
                      const int *ids, const int *off, long long n_ids, int opportunistic, int overlapped)
 {
     // table-wise: one warp per rank for the router's first half (warp 0 is also the gate)
-    const bool meta = pl->prm.part == BLS_PART_TABLE_RR && mode != BLS_MODE_LOOKUP_ONLY;
+    const bool meta = pl->prm.part == BLS_PART_TABLE_RR && mode != BLS_MODE_LOOKUP_ONLY && !overlapped;
     bls_gate_kernel<<<1, meta ? 32 * pl->prm.P : 32, 0, pl->stream>>>(pl->prm, mode, t_last, forced_floor, k, ids, off, n_ids, opportunistic, overlapped);
 }
 

@@ -37,6 +37,7 @@ def make_plan(w, tabs, k_max, cap=None):
         cap = int(cap * 1.25) + 16
     plan = bls.bls_plan(tabs, w.partition, w.P, w.local_batch, k_max, cap)
     bls.bls_set_poison(plan, True)          # every bag must be written: an unwritten one would show up as NaN
+    bls.bls_set_overlap(plan, 1)            # test workloads are small: use the overlapped mode wherever it applies
     return plan
 
 
