@@ -116,22 +116,22 @@ __device__ __forceinline__ void tile_ends(const BlsParams &p, const RouteCtx &c,
 
 // grid (NT, P), 128 threads: per-tile histogram over destinations (a tile is p.tile_bags
 // bags of one table of one requester, up to a whole chunk).  The tile's IDs are read 2048
-// at a time; the next 2048 are requested before the current ones are counted.  Lanes with
-// the same destination are counted together (one shared-memory atomic per distinct
-// destination and warp step).
+// at a time; the next 2048 are requested before the current ones are counted.  Every
+// lookup is one shared-memory atomic on its warp's own histogram (measured: much cheaper
+// than finding the lanes with equal destinations by a warp match first).
 #define BLS_RW_PER_THREAD 16
 #define BLS_RW_CHUNK (BLS_RW_PER_THREAD * BLS_ROUTE_TB)
 __global__ void __launch_bounds__(BLS_ROUTE_TB, 8) bls_rw_count_kernel(BlsParams p)
 {
-    __shared__ int cnt[BLS_MAX_RANKS];
+    __shared__ int wcnt[BLS_ROUTE_TB / 32][BLS_MAX_RANKS];     // one histogram per warp
     const int src = blockIdx.y;
     RouteCtx c;
     if (!route_ctx(p, src, c)) return;
-    const int tid = threadIdx.x, lane = tid & 31;
+    const int tid = threadIdx.x;
     const int t = blockIdx.x / p.tiles_per_table;
     const int s0 = (blockIdx.x - t * p.tiles_per_table) * p.tile_bags;
     const int nb = min(p.tile_bags, p.b - s0);
-    if (tid < BLS_MAX_RANKS) cnt[tid] = 0;
+    (&wcnt[0][0])[tid] = 0;
     int lo, hi;
     tile_ends(p, c, ((long long)src * p.T + t) * p.b + s0, nb, lo, hi);
     const unsigned rows = (unsigned)p.tab[t].rows;
@@ -154,16 +154,11 @@ __global__ void __launch_bounds__(BLS_ROUTE_TB, 8) bls_rw_count_kernel(BlsParams
         #pragma unroll
         for (int q = 0; q < BLS_RW_PER_THREAD; q++) {
             const int l = l0 + q * BLS_ROUTE_TB + tid;
-            if (l - lane < hi) {                            // same for the whole warp
-                int d = 64 + lane;                          // no lookup: matches nobody
-                if (l < hi) {
-                    unsigned id = (unsigned)cur[q];
-                    if (id >= rows) { id = 0; bad = true; }
-                    int local;
-                    d = owner_of_row(id, blk, magic, local);
-                }
-                const unsigned same = __match_any_sync(0xffffffffu, d);
-                if (l < hi && lane == __ffs(same) - 1) atomicAdd(&cnt[d], __popc(same));
+            if (l < hi) {
+                unsigned id = (unsigned)cur[q];
+                if (id >= rows) { id = 0; bad = true; }
+                int local;
+                atomicAdd(&wcnt[tid >> 5][owner_of_row(id, blk, magic, local)], 1);
             }
         }
         #pragma unroll
@@ -172,8 +167,9 @@ __global__ void __launch_bounds__(BLS_ROUTE_TB, 8) bls_rw_count_kernel(BlsParams
     if (bad) flag(p, BLS_ST_ERANGE);
     __syncthreads();
     if (tid < p.P) {
-        p.tile_cnt[((size_t)src * p.NT + blockIdx.x) * p.P + tid] = cnt[tid];
-        if (cnt[tid]) atomicAdd(&p.rw_total[src * p.P + tid], cnt[tid]);
+        const int n = wcnt[0][tid] + wcnt[1][tid] + wcnt[2][tid] + wcnt[3][tid];
+        p.tile_cnt[((size_t)src * p.NT + blockIdx.x) * p.P + tid] = n;
+        if (n) atomicAdd(&p.rw_total[src * p.P + tid], n);
     }
 }
 
@@ -241,7 +237,7 @@ __global__ void __launch_bounds__(128, 16) bls_rw_scan_kernel(BlsParams p)
 // grid (NT, P), 128 threads: places the lookups of one tile and writes its sub-bag starts.
 // The tile's lookups are classified BLS_RW_CHUNK at a time, one thread per lookup
 // (coalesced).  For every destination d a bit mask over the chunk's lookups is built
-// from warp matches (bit i set: lookup i goes to d) together with the number of set bits
+// with shared-memory atomics (bit i set: lookup i goes to d) together with the number of set bits
 // before each 32-bit word.  Everything else is a rank query on those masks:
 //   position of lookup i       = base[d] + set bits of d's mask below i   (stable by construction)
 //   start of sub-bag (bag s, d) = base[d] + set bits of d's mask below the bag's first lookup
@@ -319,15 +315,13 @@ __global__ void __launch_bounds__(BLS_ROUTE_TB, 8) bls_rw_scatter_kernel(BlsPara
         }
         #pragma unroll 1
         for (int i = tid; i - lane < nc; i += BLS_ROUTE_TB) {           // the bound is the same for a whole warp
-            int d = 64 + lane;                                          // no lookup: matches nobody
-            if (i < nc) {
-                int local;
-                d = owner_of_row((unsigned)s_id[i], blk, magic, local);
-            }
             if (lane < p.P) s_mp[lane][i >> 5].x = 0u;
             __syncwarp();
-            const unsigned same = __match_any_sync(0xffffffffu, d);
-            if (i < nc && lane == __ffs(same) - 1) s_mp[d][i >> 5].x = same;
+            if (i < nc) {
+                int local;
+                const int d = owner_of_row((unsigned)s_id[i], blk, magic, local);
+                atomicOr(&s_mp[d][i >> 5].x, 1u << lane);                // measured: far cheaper than a warp match
+            }
         }
         __syncthreads();
         // set bits before every word, one warp per destination (two words per lane)
