@@ -344,25 +344,31 @@ __global__ void __launch_bounds__(BLS_ROUTE_TB, 8) bls_rw_scatter_kernel(BlsPara
             const int d = owner_of_row((unsigned)s_id[i], blk, magic, local);
             const uint2 mp = s_mp[d][i >> 5];
             const int pos = s_base[d] + (int)mp.y + __popc(mp.x & lt);
-            if (pos < p.cap) c.sendbuf[pos] = local;
+            if (pos < p.cap) c.sendbuf[pos] = local;    // measured: grouping in shared memory first is slower
         }
-        // sub-bag starts of those bags: one thread per bag; the word and the bit mask of the
-        // rank query are the same for all destinations, and a bag's P entries are contiguous
-        // in the bag-major layout
-        for (int s = s_lo + tid; s < s_hi; s += BLS_ROUTE_TB) {
-            const int x = min(max(s_off[s] - c0, 0), nc);
-            const int wd = x >> 5;
-            const unsigned below = (1u << (x & 31)) - 1u;
-            auto start_of = [&](int d) {
-                const uint2 mp = s_mp[d][wd];
-                return min(s_base[d] + (int)mp.y + __popc(mp.x & below), p.cap);
-            };
-            int *row = rows_out + (size_t)s * p.P;
-            if ((p.P & 3) == 0) {
-                for (int d = 0; d < p.P; d += 4)
-                    *reinterpret_cast<int4 *>(row + d) = make_int4(start_of(d), start_of(d + 1), start_of(d + 2), start_of(d + 3));
-            } else {
-                for (int d = 0; d < p.P; d++) row[d] = start_of(d);
+        // sub-bag starts of those bags (a bag's P entries are contiguous in the bag-major
+        // layout).  P a multiple of 4: one thread per four destinations of a bag, so that a
+        // warp's 16-byte stores cover one contiguous piece of the array; else one thread per entry.
+        if ((p.P & 3) == 0) {
+            const int qpb = p.P >> 2;                           // 16-byte pieces per bag
+            for (int e = tid; e < (s_hi - s_lo) * qpb; e += BLS_ROUTE_TB) {
+                const int s = s_lo + e / qpb, d = (e % qpb) * 4;
+                const int x = min(max(s_off[s] - c0, 0), nc);
+                const int wd = x >> 5;
+                const unsigned below = (1u << (x & 31)) - 1u;
+                auto start_of = [&](int dd) {
+                    const uint2 mp = s_mp[dd][wd];
+                    return min(s_base[dd] + (int)mp.y + __popc(mp.x & below), p.cap);
+                };
+                *reinterpret_cast<int4 *>(rows_out + (size_t)s * p.P + d) =
+                    make_int4(start_of(d), start_of(d + 1), start_of(d + 2), start_of(d + 3));
+            }
+        } else {
+            for (int e = tid; e < (s_hi - s_lo) * p.P; e += BLS_ROUTE_TB) {
+                const int s = s_lo + e / p.P, d = e % p.P;
+                const int x = min(max(s_off[s] - c0, 0), nc);
+                const uint2 mp = s_mp[d][x >> 5];
+                rows_out[(size_t)s * p.P + d] = min(s_base[d] + (int)mp.y + __popc(mp.x & ((1u << (x & 31)) - 1u)), p.cap);
             }
         }
         s_lo = s_hi;
