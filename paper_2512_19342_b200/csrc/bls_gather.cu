@@ -310,7 +310,7 @@ bls_gather_hot_kernel(BlsParams p, int R, int runs_per_chunk)
 // order inside registers and the pooled vector is stored once.  No atomics, no
 // zero-filled output, and the result does not depend on timing.
 template <int LANES, int DT>
-__global__ void __launch_bounds__(256, 3)
+__global__ void __launch_bounds__(256, 4)
 bls_gather_rowwise_kernel(BlsParams p, int R, int runs_per_chunk, int n_runs)
 {
     constexpr int GPW = 32 / LANES;
@@ -494,9 +494,11 @@ static void launch_gather(const bls_plan_t *pl)
     const int rpc = (p.b + R - 1) / R;
     // table-wise: runs of sub-bags of one (owner, table, requester); row-wise: runs of bags of one (table, requester)
     const long long n_runs = (long long)(rowwise ? p.T : p.NI) * p.P * rpc;
-    // persistent blocks: as many as stay resident (3 per SM at 80 registers), fewer for small workloads
+    // persistent blocks: as many as stay resident (table-wise: 3 per SM at 80 registers; row-wise: 4 at 64
+    // registers, measured faster than 3 or 5), fewer for small workloads
     const long long want = (n_runs + 8 * (32 / LANES) - 1) / (8 * (32 / LANES));
-    const int blocks = (int)(want < 1 ? 1 : (want > pl->sm_count * 3 ? pl->sm_count * 3 : want));
+    const int per_sm = rowwise ? 4 : 3;
+    const int blocks = (int)(want < 1 ? 1 : (want > pl->sm_count * per_sm ? pl->sm_count * per_sm : want));
     if (rowwise) {
         bls_gather_rowwise_kernel<LANES, DT><<<blocks, 256, 0, pl->stream>>>(p, R, rpc, (int)n_runs);
     } else if (p.hot.enabled) {
