@@ -182,8 +182,8 @@ bls_status_t bls_a2a_post(bls_a2a_t *h, const void *sendbuf, int64_t send_stride
     a.rdispls = h->rdispls + (size_t)slot * h->P * h->P;
     a.arrived = h->arrived + (size_t)slot * h->P;
     a.status = h->status; a.blocks_done = h->blocks_done;
-    // enough chunks to fill the machine, at least 16 KiB each
-    long long chunks = ((long long)h->sm_count * 8 + h->P * h->P - 1) / (h->P * h->P);
+    // four times as many chunks as fill the machine (measured: evens out the tail on large messages), at least 16 KiB each
+    long long chunks = ((long long)h->sm_count * 32 + h->P * h->P - 1) / (h->P * h->P);
     long long chunk_bytes = (max_segment_bytes + chunks - 1) / (chunks > 0 ? chunks : 1);
     if (chunk_bytes < 16384) chunk_bytes = 16384;
     chunk_bytes = (chunk_bytes + 15) / 16 * 16;
