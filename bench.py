@@ -153,17 +153,18 @@ def capacity(w, inputs):
 
 
 def traffic_record(kernel_src: str, workload_name: str):
-    """DRAM bytes per launch of the gather kernel from the committed ncu capture,
-    or None when the kernel source has changed since the counters were taken."""
-    path = os.path.join(ROOT, "profiles", "gather_pool_traffic.json")
+    """DRAM bytes per launch of the gather kernel from the committed ncu captures
+    (profiles/gather_traffic.json, one record per workload), or None when there is no
+    record for this workload or the kernel source has changed since the counters were taken."""
+    path = os.path.join(ROOT, "profiles", "gather_traffic.json")
     if not os.path.exists(path):
         return None
     try:
         rec = json.load(open(path))
         digest = hashlib.sha256(open(kernel_src, "rb").read()).hexdigest()
-        if rec.get("kernel_sha256") != digest or rec.get("workload") != workload_name:
+        if rec.get("kernel_sha256") != digest:
             return None
-        return float(rec["dram_bytes_per_launch"])
+        return float(rec["records"][workload_name]["dram_bytes_per_launch"])
     except Exception:
         return None
 
@@ -193,16 +194,28 @@ def host_tables_for_oracle(w, cores):
 def oracle_iteration(w, data, ids, off, cores):
     import oracle
     oracle.route(w.P, w.T, w.local_batch, w.partition, [t.rows for t in w.tables], ids, off, nthreads=cores)
-    oracle.pool_definition(w.P, w.T, w.local_batch, w.tables, data, ids, off, nthreads=cores)
+    return oracle.pool_definition(w.P, w.T, w.local_batch, w.tables, data, ids, off, nthreads=cores)
 
 
-def cpu_baseline(w, inputs, target_s=12.0):
+def cpu_baseline(w, inputs, gpu_out0=None, target_s=12.0):
+    """Times the oracle on a bounded sample of the workload.  The oracle's pooled output of the
+    first timed batch (computed outside the timed region) is also compared, vector by vector, with
+    what the CUDA path produced for the same batch: returns (baseline, parity)."""
+    import oracle
     cores = len(os.sched_getaffinity(0))
     data, how = host_tables_for_oracle(w, cores)
     ids, off = inputs[0]
     t0 = time.perf_counter()
-    oracle_iteration(w, data, ids, off, cores)
+    want0 = oracle_iteration(w, data, ids, off, cores)
     t1 = time.perf_counter() - t0
+    parity = None
+    if gpu_out0 is not None:
+        tol = 1e-5 if w.tables[0].dtype == "f32" else 1e-2
+        err = oracle.vector_rel_err(gpu_out0, want0)
+        parity = {"max_rel_err": err, "tolerance": tol, "ok": bool(err <= tol), "vectors": int(w.n_bags),
+                  "what": "every pooled vector of the first timed batch, CUDA path (bls_step, bound 0) against the "
+                          "oracle's fp64 sum by definition; per vector max|g-o| / max|o|, maximised over vectors"}
+    del want0
     n = int(max(1, min(400, round(target_s / max(t1, 1e-3)))))
     lookups = 0
     t0 = time.perf_counter()
@@ -213,7 +226,7 @@ def cpu_baseline(w, inputs, target_s=12.0):
     dt = time.perf_counter() - t0
     return {"value": lookups / dt, "unit": "lookups/s", "cores": cores, "kind": "oracle",
             "sample": f"{n} full iteration(s) of {w.name} ({lookups} lookups, {dt:.1f} s): route + fp64 pooling by "
-                      f"definition, one OpenMP thread per core; {how}"}
+                      f"definition, one OpenMP thread per core; {how}"}, parity
 
 
 def run_reference(args):
@@ -364,6 +377,12 @@ def run_mine(args):
     st, _ = bls.bls_status(plan)
     if st != bls.BLS_OK:
         raise RuntimeError(f"device status {st} after warm-up")
+    # the CUDA path's answer to the first timed batch, kept for the comparison with the oracle
+    gpu_out0 = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        out0, _ = bls.bls_step(plan, 0, *d_in[0])
+        gpu_out0 = out0.cpu().numpy()
+        del out0
 
     sampler = ClockSampler(local_rank) if rank == 0 else None
     units = float(sum(Ls[t % nd] for t in range(args.steps)))
@@ -482,6 +501,8 @@ def run_mine(args):
     step_bytes, gather_bytes = algorithmic_bytes(w, L_mean)
     ms_gather = prof["ms_gather"] / max(1, prof["calls"])
     ach = gather_bytes / (ms_gather * 1e-3) / 1e9
+    traffic = traffic_record(os.path.join(ROOT, "paper_2512_19342_b200", "csrc", "bls_gather.cu"), w.name)
+    dram_gbs = None if traffic is None else traffic / (ms_gather * 1e-3) / 1e9
     step_gbs = step_bytes * world / (ms_head / args.steps * 1e-3) / 1e9
     result = {
         "metric": "embedding_lookups_per_s", "value": tot_head / (ms_head * 1e-3), "unit": "lookups/s",
@@ -502,8 +523,11 @@ def run_mine(args):
                           "bytes_per_step": step_bytes, "peak_source": peak_src},
         "roofline": {"bound": "hbm", "kernel": gather_kernel, "achieved": ach, "peak": peak, "unit": "GB/s",
                      "frac": ach / peak, "frac_of_nominal_8TBs": ach / NOMINAL_HBM_GBS,
-                     "traffic": traffic_record(os.path.join(ROOT, "paper_2512_19342_b200", "csrc", "bls_gather.cu"), w.name),
-                     "bytes_per_launch": gather_bytes, "ms_per_launch": ms_gather, "peak_source": peak_src},
+                     "traffic": traffic, "dram_achieved": dram_gbs,
+                     "dram_frac": None if dram_gbs is None else dram_gbs / peak,
+                     "bytes_per_launch": gather_bytes, "ms_per_launch": ms_gather, "peak_source": peak_src,
+                     "note": "frac counts algorithmic bytes (every row of every lookup, also those served by L1/L2); "
+                             "dram_frac counts the DRAM bytes ncu measured for one launch (traffic) over the same time"},
         "roofline_uniform_ids": None if uniform is None else {
             "bound": "hbm", "kernel": gather_kernel, "achieved": uniform["achieved"], "peak": peak,
             "unit": "GB/s", "frac": uniform["achieved"] / peak, "ms_per_launch": uniform["ms_per_launch"],
@@ -516,7 +540,9 @@ def run_mine(args):
         "clocks": clocks, "e2e": e2e, "gpu_launches": launches, "delay_sweep": delay_sweep, "straggler": straggler,
     }
     if not args.no_cpu_baseline and world == 1:
-        result["cpu_baseline"] = cpu_baseline(w, inputs)
+        result["cpu_baseline"], result["parity"] = cpu_baseline(w, inputs, gpu_out0)
+        if result["parity"] is not None:
+            result["parity_max_rel_err"] = result["parity"]["max_rel_err"]
     print(json.dumps(result))
 
 

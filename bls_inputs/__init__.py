@@ -63,7 +63,7 @@ class Workload:
     lengths: str                # "one" | "poisson20c" | "poisson10" | "pareto15c" | "mixed"
     id_dist: str                # "uniform" | "zipf"
     zipf_s: float
-    hot_placement: bool         # hot rows of tables 0..7 placed in the first two row blocks
+    hot_ranges: Tuple[Tuple[int, int], ...]   # tables 0..7: the hottest rows land alternately in these row ranges; () = anywhere
     iterations: int
     ks: Tuple[int, ...]
     seed: int
@@ -104,29 +104,33 @@ def workload(number: int, rows_scale: float = 1.0, batch_scale: float = 1.0) -> 
         P = 4
         tables = _specs([rs(10_000)] * 8, 16, "f32", "normal", 0)
         return Workload("cfg1_onehot_8x10k_d16", 1, tables, P, "table_rr", bs(256, P),
-                        "one", "uniform", 0.0, False, 10, (0, 2), 1000)
+                        "one", "uniform", 0.0, (), 10, (0, 2), 1000)
     if number == 2:
         P = 8
         rng = np.random.Generator(np.random.PCG64(2001))
         rows = np.floor(10.0 ** rng.uniform(3.0, 6.0, size=26)).astype(np.int64)
         tables = _specs([rs(r) for r in rows], 16, "f32", "normal", 2000)
         return Workload("cfg2_onehot_26xlogu_d16", 2, tables, P, "table_rr", bs(2048, P),
-                        "one", "uniform", 0.0, False, 100, (0, 1, 4), 2000)
+                        "one", "uniform", 0.0, (), 100, (0, 1, 4), 2000)
     if number == 3:
         P = 8
         tables = _specs([rs(1_000_000)] * 26, 64, "f32", "hash", 3000)
         return Workload("cfg3_zipf_multihot_26x1m_d64", 3, tables, P, "table_rr", bs(16384, P),
-                        "poisson20c", "zipf", 1.05, False, 100, (0, 1, 4), 3000)
+                        "poisson20c", "zipf", 1.05, (), 100, (0, 1, 4), 3000)
     if number == 4:
         P = 16
-        tables = _specs([rs(2_000_000)] * 64, 128, "bf16", "hash", 4000)
+        n = rs(2_000_000)
+        tables = _specs([n] * 64, 128, "bf16", "hash", 4000)
+        # "the 8 hottest tables' hot rows placed on 2 ranks": the first and the second sixteenth of the rows
+        sixteenth = max(1, n // 16)
         return Workload("cfg4_unbalanced_rowwise_64x2m_d128_bf16", 4, tables, P, "row_block",
-                        bs(32768, P), "poisson10", "zipf", 1.2, True, 200, (0, 1, 2, 8), 4000)
+                        bs(32768, P), "poisson10", "zipf", 1.2,
+                        ((0, sixteenth), (sixteenth, min(n, 2 * sixteenth))), 200, (0, 1, 2, 8), 4000)
     if number == 5:
         P = 32
         tables = _specs([rs(5_000_000)] * 100, 64, "f16", "hash", 5000)
         return Workload("cfg5_large_100x5m_d64_f16", 5, tables, P, "table_rr", bs(65536, P),
-                        "pareto15c", "zipf", 1.1, False, 100, (4,), 5000)
+                        "pareto15c", "zipf", 1.1, (), 100, (4,), 5000)
     raise ValueError("workload number must be 1..5")
 
 
@@ -136,7 +140,7 @@ def tiny_workload(T=3, P=2, b=2, rows=7, dim=4, dtype="f32", partition="table_rr
     rows_l = rows if isinstance(rows, (list, tuple)) else [rows] * T
     tables = _specs(rows_l, dim, dtype, "normal", seed)
     return Workload(f"tiny_T{T}_P{P}_b{b}", 0, tables, P, partition, b, lengths, id_dist,
-                    zipf_s, False, 4, (0, 1, 2), seed)
+                    zipf_s, (), 4, (0, 1, 2), seed)
 
 
 # --------------------------------------------------------------------------
@@ -229,9 +233,9 @@ _cdf_cache: dict = {}
 def table_permutation(w: Workload, t: int) -> np.ndarray:
     """Random map from popularity rank (0 = hottest) to row number for table t.
 
-    For the unbalanced shape, tables 0..7 place popularity ranks 0..4095
-    alternately into the first and the second of the P equal row blocks; every
-    other rank/table is uniformly random.
+    When the workload names row ranges for its hot rows (``hot_ranges``, two of
+    them), tables 0..7 place popularity ranks 0..4095 alternately into the first
+    and the second range; every other rank/table is uniformly random.
     """
     key = (w.name, w.tables[t].rows, t, w.seed)
     if key in _perm_cache:
@@ -239,14 +243,14 @@ def table_permutation(w: Workload, t: int) -> np.ndarray:
     n = w.tables[t].rows
     rng = np.random.Generator(np.random.PCG64([w.seed, 1, t]))
     perm = rng.permutation(n).astype(np.int32)
-    if w.hot_placement and t < 8:
-        blk = -(-n // w.P)
-        nhot = min(4096, n // 4, 2 * blk)
-        if nhot >= 2:
-            # positions (rows) the hot ranks must land on: alternate block 0 / block 1
+    if len(w.hot_ranges) == 2 and t < 8:
+        (lo0, hi0), (lo1, hi1) = w.hot_ranges
+        nhot = min(4096, n // 4, (hi0 - lo0) + (hi1 - lo1))
+        if nhot >= 2 and hi1 > lo1:
+            # positions (rows) the hot ranks must land on: alternate first range / second range
             half = (nhot + 1) // 2
-            r0 = rng.choice(min(blk, n), size=half, replace=False)
-            r1 = blk + rng.choice(max(1, min(blk, n - blk)), size=nhot - half, replace=False)
+            r0 = lo0 + rng.choice(hi0 - lo0, size=half, replace=False)
+            r1 = lo1 + rng.choice(hi1 - lo1, size=nhot - half, replace=False)
             target = np.empty(nhot, dtype=np.int64)
             target[0::2] = r0
             target[1::2] = r1[: len(target[1::2])]

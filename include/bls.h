@@ -163,7 +163,8 @@ bls_status_t bls_step_host(bls_plan_t *plan, int k, const int32_t *ids /*host*/,
                            float *host_out /*host*/, int64_t *out_iter /*host out*/);
 bls_status_t bls_drain_host(bls_plan_t *plan, float *host_out /*host*/, int64_t *out_iter /*host out*/);
 
-/* ---- inspection ---- */
+/* ---- inspection (bls_view, bls_counters, bls_status, bls_set_poison, bls_set_wait_limit,
+ * bls_profile*, bls_set_tuning: debugging and measurement aids with no counterpart in the paper) ---- */
 /* Device pointers of the slot that holds iteration `iter` (must still be in the ring). */
 bls_status_t bls_view(bls_plan_t *plan, int64_t iter, bls_route_view_t *view /*host out*/);
 /* Synchronises the stream; copies the P per-rank counters to host arrays (may be NULL). */
@@ -261,7 +262,12 @@ bls_status_t bls_fill_hash_table(void *weight, int64_t rows, int32_t dim, int32_
  * outstanding (BLS_ESTATE otherwise): k_max = 0 is a plain alltoallv.
  *   workspace        device, 256-byte aligned, bls_a2a_bytes() long, borrowed
  *   sendbuf/sendcounts/sdispls  device; counts and displacements are int64 [P][P] in bytes
- *   max_segment_bytes host hint: the largest sendcounts entry (sizes the launch)
+ *   max_segment_bytes host hint: the largest sendcounts entry.  It only sizes the launch:
+ *                    a segment longer than the hint is still copied whole
+ * A segment whose count or displacement leaves the sender's stride (BLS_EINVAL), or that no
+ * longer fits behind the accepted segments of lower-ranked sources in the receiver's buffer
+ * (BLS_ENOSPC), is rejected: it arrives as an empty segment (recvcounts 0), the receiver
+ * counts one message fewer, and bls_a2a_wait's check then also latches BLS_ESTATE.
  * Asynchronous on the stream; device-detected conditions (segment outside the send
  * stride: BLS_EINVAL, receive capacity exceeded: BLS_ENOSPC) via bls_a2a_status, which
  * synchronises. */
@@ -293,8 +299,8 @@ bls_status_t bls_a2a_status(bls_a2a_t *handle);
  *   sendcounts, sdispls  device out, int32 [P][P] indexed [src][dst]
  *   sendbuf     device out, int32 [P][cap]: rank src's packed send buffer at src*cap
  *   sub_start   device out, int32 [P][T*local_batch + 1], ordered (dst, table, sample)
- *   status      device out, one int32: 0, or an OR of 1 (malformed offsets),
- *               2 (cap too small), 4 (ID out of range, replaced by row 0)
+ *   status      device out, one int32: 0, or an OR of 1 (malformed offsets or a table
+ *               height below 1), 2 (cap too small), 4 (ID out of range, replaced by row 0)
  * Results are identical to bls_route + bls_view on a table-wise plan.
  *
  * Limits and rules: P * (T + 1) <= 32768, else BLS_ENOSPC.  The first call on a

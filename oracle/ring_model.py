@@ -101,9 +101,10 @@ class RingModel:
 
     def _note(self, ev):
         self.trace.append(ev)
-        # "any two processes may be in iterations i and j as long as |j - i| <= k":
-        # the fastest rank is inside the newest iteration it has posted, the
-        # slowest is still inside the oldest iteration not yet completed.
+        # Section III (definition of the bound k): the iterations two ranks are
+        # working on never differ by more than k.  The fastest rank is inside the
+        # newest iteration it has posted, the slowest is still inside the oldest
+        # iteration not yet completed.
         self.max_spread = max(self.max_spread, max(self.posted) - 1 - min(self.done))
 
     def finished(self):

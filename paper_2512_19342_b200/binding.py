@@ -13,7 +13,7 @@ from typing import List, Optional, Sequence, Tuple
 import torch
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.environ.get("BLS_LIBRARY", os.path.join(_HERE, "libbls.so"))   # override: an alternative build
+LIB_PATH = os.path.join(_HERE, "libbls.so")
 
 BLS_OK, BLS_EINVAL, BLS_ENOSPC, BLS_ECUDA, BLS_ERANGE, BLS_ETIMEOUT, BLS_ESTATE = range(7)
 BLS_F32, BLS_BF16, BLS_F16 = 0, 1, 2

@@ -61,43 +61,65 @@ struct A2aArgs {
     int *status, *blocks_done;
 };
 
-// grid (chunks, P*P): block (c, src*P+dst) copies chunk c of the segment src -> dst.
+// Whether the segment src -> dst is accepted, and where it lands.  Receiver dst takes the
+// segments of sources 0, 1, ... in rank order: a segment is accepted when its count and
+// displacement lie inside the sender's stride and it still fits behind the accepted
+// segments of the lower-ranked sources; a rejected one counts as empty, so the reported
+// counts and displacements always agree with each other.
+__device__ __forceinline__ bool a2a_accept(const A2aArgs &a, int src, int dst, long long &n, long long &rd, int &why)
+{
+    rd = 0;
+    bool ok = false;
+    for (int s2 = 0; s2 <= src; s2++) {
+        n = a.sendcounts[s2 * a.P + dst];
+        const long long sd = a.sdispls[s2 * a.P + dst];
+        const bool inside = n >= 0 && sd >= 0 && sd + n <= a.send_stride;
+        ok = inside && rd + n <= a.cap;
+        why = inside ? BLS_ST_ENOSPC : BLS_ST_EINVAL;
+        if (s2 < src && ok) rd += n;
+    }
+    return ok;
+}
+
+// grid (chunks, P*P): the blocks (*, src*P+dst) copy the segment src -> dst, chunk by chunk
+// with stride gridDim.x, so a segment of any length is covered whatever the host's size hint was.
 __global__ void __launch_bounds__(256) bls_a2a_put_kernel(A2aArgs a, long long chunk_bytes)
 {
     const int src = blockIdx.y / a.P, dst = blockIdx.y % a.P;
-    const long long n = a.sendcounts[src * a.P + dst];
-    long long rd = 0;                                     // rdispls[dst][src]: counts of lower-ranked sources
-    for (int s2 = 0; s2 < src; s2++) rd += max(a.sendcounts[s2 * a.P + dst], 0LL);
-    const long long sd = a.sdispls[src * a.P + dst];
-    bool ok = n >= 0 && sd >= 0 && sd + n <= a.send_stride && rd + n <= a.cap;
-    if (!ok && blockIdx.x == 0 && threadIdx.x == 0)
-        atomicOr(a.status, (n < 0 || sd < 0 || sd + n > a.send_stride) ? BLS_ST_EINVAL : BLS_ST_ENOSPC);
+    long long n, rd;
+    int why;
+    const bool ok = a2a_accept(a, src, dst, n, rd, why);
     if (blockIdx.x == 0 && threadIdx.x == 0) {
+        if (!ok) atomicOr(a.status, why);
         a.recvcounts[dst * a.P + src] = ok ? n : 0;
         a.rdispls[dst * a.P + src] = rd;
     }
     if (ok) {
-        const char *from = a.send + (size_t)src * a.send_stride + sd;
+        const char *from = a.send + (size_t)src * a.send_stride + a.sdispls[src * a.P + dst];
         char *to = a.recv + (size_t)dst * a.cap + rd;
-        const long long lo = (long long)blockIdx.x * chunk_bytes, hi = min(n, lo + chunk_bytes);
-        if (((reinterpret_cast<uintptr_t>(from) | reinterpret_cast<uintptr_t>(to)) & 15) == 0) {
-            const long long v_hi = lo + ((hi - lo) & ~15LL);          // 16 bytes per thread while both sides are aligned
-            long long i = lo + (long long)threadIdx.x * 16;
-            for (; i + 3 * 256 * 16 < v_hi; i += 4 * 256 * 16) {       // four loads in flight per thread
-                uint4 v[4];
-                #pragma unroll
-                for (int q = 0; q < 4; q++) v[q] = __ldcs(reinterpret_cast<const uint4 *>(from + i + q * 256 * 16));
-                #pragma unroll
-                for (int q = 0; q < 4; q++) __stcs(reinterpret_cast<uint4 *>(to + i + q * 256 * 16), v[q]);
+        const bool aligned = ((reinterpret_cast<uintptr_t>(from) | reinterpret_cast<uintptr_t>(to)) & 15) == 0;
+        for (long long lo = (long long)blockIdx.x * chunk_bytes; lo < n; lo += (long long)gridDim.x * chunk_bytes) {
+            const long long hi = min(n, lo + chunk_bytes);
+            if (aligned) {
+                const long long v_hi = lo + ((hi - lo) & ~15LL);          // 16 bytes per thread while both sides are aligned
+                long long i = lo + (long long)threadIdx.x * 16;
+                for (; i + 3 * 256 * 16 < v_hi; i += 4 * 256 * 16) {       // four loads in flight per thread
+                    uint4 v[4];
+                    #pragma unroll
+                    for (int q = 0; q < 4; q++) v[q] = __ldcs(reinterpret_cast<const uint4 *>(from + i + q * 256 * 16));
+                    #pragma unroll
+                    for (int q = 0; q < 4; q++) __stcs(reinterpret_cast<uint4 *>(to + i + q * 256 * 16), v[q]);
+                }
+                for (; i < v_hi; i += 256 * 16)
+                    *reinterpret_cast<uint4 *>(to + i) = __ldcs(reinterpret_cast<const uint4 *>(from + i));
+                for (long long i2 = v_hi + threadIdx.x; i2 < hi; i2 += 256) to[i2] = from[i2];
+            } else {
+                for (long long i = lo + threadIdx.x; i < hi; i += 256) to[i] = from[i];
             }
-            for (; i < v_hi; i += 256 * 16)
-                *reinterpret_cast<uint4 *>(to + i) = __ldcs(reinterpret_cast<const uint4 *>(from + i));
-            for (long long i = v_hi + threadIdx.x; i < hi; i += 256) to[i] = from[i];
-        } else {
-            for (long long i = lo + threadIdx.x; i < hi; i += 256) to[i] = from[i];
         }
     }
-    // the last block to finish counts the arrivals: one message per source at every receiver
+    // the last block to finish counts the arrivals: at every receiver one message per source
+    // whose segment was accepted (all copies are complete by then)
     __shared__ int s_last;
     __syncthreads();
     if (threadIdx.x == 0) {
@@ -106,12 +128,22 @@ __global__ void __launch_bounds__(256) bls_a2a_put_kernel(A2aArgs a, long long c
     }
     __syncthreads();
     if (s_last) {
-        if ((int)threadIdx.x < a.P) atomicAdd(&a.arrived[threadIdx.x], a.P);
+        if ((int)threadIdx.x < a.P) {
+            int got = 0;
+            for (int s2 = 0; s2 < a.P; s2++) {
+                long long n2, rd2;
+                int why2;
+                got += a2a_accept(a, s2, threadIdx.x, n2, rd2, why2) ? 1 : 0;
+            }
+            atomicAdd(&a.arrived[threadIdx.x], got);
+        }
         if (threadIdx.x == 0) *a.blocks_done = 0;
     }
 }
 
-// Completion check of the oldest request: every receiver of the slot has counted P messages.
+// Completion check of the oldest request: every receiver of the slot has counted P messages
+// (fewer means a segment was rejected, which the post has already reported, or that the
+// slot was completed before its request had run).
 __global__ void bls_a2a_complete_kernel(int *arrived, int P, int *status)
 {
     const int r = threadIdx.x;

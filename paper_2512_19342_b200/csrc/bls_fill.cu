@@ -38,7 +38,11 @@ extern "C" bls_status_t bls_fill_hash_table(void *weight, int64_t rows, int32_t 
     if (!weight || rows < 1 || dim < 1 || dim > 65536 || t < 0 || t > 65535 || rows > 0xffffffffLL) return BLS_EINVAL;
     long long n = (long long)rows * dim;
     long long blocks = (n + 255) / 256;
-    if (blocks > 148 * 32) blocks = 148 * 32;
+    int dev = 0, sms = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess ||
+        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms < 1)
+        return BLS_ECUDA;
+    if (blocks > (long long)sms * 32) blocks = (long long)sms * 32;   // grid-stride loop: 32 blocks per SM at most
     cudaStream_t s = (cudaStream_t)cuda_stream;
     if (dtype == BLS_F32) bls_fill_kernel<BLS_F32><<<(unsigned)blocks, 256, 0, s>>>(weight, rows, dim, seed, t);
     else if (dtype == BLS_BF16) bls_fill_kernel<BLS_BF16><<<(unsigned)blocks, 256, 0, s>>>(weight, rows, dim, seed, t);

@@ -92,12 +92,18 @@ __global__ void __launch_bounds__(128) bls_static_meta_kernel(StaticArgs a)
         int i = 0;
         for (int d = 0; d < a.P; d++) {
             const int nt = d < a.T ? (a.T - d + a.P - 1) / a.P : 0;
-            a.sdispls[src * a.P + d] = (int)run;
+            // totals beyond the 32-bit range are clamped (and reported below as exceeding cap), so
+            // that no chunk base can wrap to a negative position
+            a.sdispls[src * a.P + d] = (int)min(run, (long long)0x7fffffff);
             const long long before = run;
-            for (int q = 0; q < nt; q++, i++) { const int n = cb[i]; cb[i] = (int)run; run += n; }
-            a.sendcounts[src * a.P + d] = (int)(run - before);
+            for (int q = 0; q < nt; q++, i++) {
+                const int n = cb[i];
+                cb[i] = (int)min(run, (long long)0x7fffffff);
+                run += n;
+            }
+            a.sendcounts[src * a.P + d] = (int)min(run - before, (long long)0x7fffffff);
         }
-        cb[a.T] = (int)run;
+        cb[a.T] = (int)min(run, (long long)0x7fffffff);
         if (run > a.cap) atomicOr(a.status, BLS_ST_ENOSPC);
         a.sub_start[(size_t)src * ((size_t)a.T * a.b + 1) + (size_t)a.T * a.b] = (int)(run > a.cap ? a.cap : run);
     }
@@ -126,13 +132,17 @@ __global__ void __launch_bounds__(256) bls_static_copy_kernel(StaticArgs a, int 
         if (threadIdx.x == nb - 1) s_hi = (int)en;
     }
     __syncthreads();
-    const unsigned long long rows = (unsigned long long)a.rows[t];
+    // a table height below 1 is malformed input: reported, and every ID of the table is then out of range
+    const long long rows_in = a.rows[t];
+    if (rows_in < 1 && threadIdx.x == 0) atomicOr(a.status, BLS_ST_EINVAL);
+    const unsigned long long rows = rows_in < 1 ? 0ull : (unsigned long long)rows_in;
     const int lo = s_lo, hi = max(s_lo, s_hi);
     int *dst = a.sendbuf + (size_t)src * a.cap;
     for (int l = lo + threadIdx.x; l < hi; l += blockDim.x) {
         int id = a.ids[off0 + l];
         if ((unsigned long long)(unsigned)id >= rows) { id = 0; atomicOr(a.status, BLS_ST_ERANGE); }
-        if (cb + l < a.cap) dst[cb + l] = id;
+        const long long pos = (long long)cb + l;
+        if (pos >= 0 && pos < a.cap) dst[pos] = id;
     }
 }
 

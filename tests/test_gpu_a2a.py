@@ -78,3 +78,34 @@ def test_ring_and_capacity_limits():
     a2a.wait()
     assert a2a.status() == bls.BLS_ENOSPC
     assert torch.ones(4, device="cuda").sum().item() == 4.0
+
+
+def test_size_hint_below_the_largest_segment_does_not_truncate():
+    """max_segment_bytes only sizes the launch: a segment longer than the hint is still copied whole."""
+    P = 4
+    rng = np.random.Generator(np.random.PCG64(77))
+    send, counts, sd = make_request(P, rng, 300_000)
+    a2a = bls.A2a(P, 0, int(counts.sum(axis=0).max()) + 64)
+    a2a.post(torch.from_numpy(send).cuda(), torch.from_numpy(counts).cuda(), torch.from_numpy(sd).cuda(), 1000)
+    recv, rc, rd, _ = a2a.wait()
+    want = expected(send, counts, sd)
+    recv = recv.cpu().numpy()
+    for d in range(P):
+        assert np.array_equal(recv[d, :len(want[d])], want[d])
+    assert np.array_equal(rc.cpu().numpy(), counts.T)
+    assert a2a.status() == bls.BLS_OK
+
+
+def test_rejected_segment_counts_as_empty():
+    """A segment that does not fit is reported, arrives nowhere, and the receive-side counts and
+    displacements stay consistent with each other."""
+    P = 2
+    a2a = bls.A2a(P, 0, 256)
+    send = torch.arange(512, dtype=torch.int32, device="cuda").to(torch.uint8).repeat(P, 1)
+    counts = torch.tensor([[100, 10], [200, 10]], dtype=torch.int64, device="cuda")   # receiver 0: 100 fits, 200 more do not
+    sd = torch.tensor([[0, 300], [0, 300]], dtype=torch.int64, device="cuda")
+    a2a.post(send, counts, sd, 200)
+    recv, rc, rd, _ = a2a.wait()
+    assert a2a.status() == bls.BLS_ENOSPC                   # the rejected segment; the completion check also sees it missing
+    assert rc.cpu().tolist() == [[100, 0], [10, 10]]
+    assert rd.cpu().tolist() == [[0, 100], [0, 10]]

@@ -14,6 +14,14 @@ from test_gpu_parity import TOL, check_route, dev_tables, make_plan
 pytestmark = pytest.mark.gpu
 
 
+def assert_matches_oracle(w, data, inputs, outs):
+    """Every handed-back iteration against the oracle's pooled output by definition."""
+    for it, (ids, off) in enumerate(inputs):
+        want = oracle.pool_definition(w.P, w.T, w.local_batch, w.tables, data, ids, off)
+        err = oracle.vector_rel_err(outs[it].cpu().numpy(), want)
+        assert err <= TOL[w.tables[0].dtype], (it, err)
+
+
 def run_loop(w, tabs, k, n_iter, k_max=None, stalls=None, check_views=False, wait_limit=None):
     """Listing 2's loop: n_iter steps then the drain; returns {iteration: output}."""
     plan = make_plan(w, tabs, k if k_max is None else k_max)
@@ -88,16 +96,19 @@ def test_delayed_ranks_lag_within_the_bound(part):
     data = [bi.table_values(t) for t in w.tables]
     tabs = dev_tables(w, data)
     n_iter = 10
-    ref, *_ = run_loop(w, tabs, 0, n_iter)
+    ref, inputs, *_ = run_loop(w, tabs, 0, n_iter)
+    assert_matches_oracle(w, data, inputs, ref)
     for k in (1, 3):
         outs, _, status, lag = run_loop(w, tabs, k, n_iter, stalls={1: 3_000_000, 2: 500_000})
         assert status == bls.BLS_OK
         assert 1 <= lag <= k, lag                                     # somebody really ran ahead
+        assert_matches_oracle(w, data, inputs, outs)
         for it in range(n_iter):
             assert torch.equal(outs[it], ref[it]), (k, it)
     # bound 0: the delay is paid every iteration, nobody runs ahead
     outs, _, status, lag = run_loop(w, tabs, 0, 4, stalls={1: 1_000_000})
     assert status == bls.BLS_OK and lag == 0
+    assert_matches_oracle(w, data, inputs[:4], outs)
     assert all(torch.equal(outs[i], ref[i]) for i in range(4))
 
 
@@ -214,7 +225,8 @@ def test_random_delays_are_masked_by_the_bound():
     before each iteration.  Bound 0 pays the largest of the P delays in every iteration;
     a bound k > 0 lets ranks drift apart and hides part of it.  Results do not change."""
     w = bi.tiny_workload(T=4, P=4, b=64, rows=500, dim=16, lengths="poisson10")
-    tabs = dev_tables(w, [bi.table_values(t) for t in w.tables])
+    data = [bi.table_values(t) for t in w.tables]
+    tabs = dev_tables(w, data)
     n_iter, span = 40, 400_000                                  # delays uniform in [0, 400 us]
     inputs = [bi.make_iteration(w, t) for t in range(n_iter)]
     d_in = [(torch.from_numpy(i).cuda(), torch.from_numpy(o).cuda()) for i, o in inputs]
@@ -241,6 +253,7 @@ def test_random_delays_are_masked_by_the_bound():
         torch.cuda.synchronize()
         status, lag = bls.bls_status(plan)
         assert status == bls.BLS_OK and lag <= k and len(got) == n_iter
+        assert_matches_oracle(w, data, inputs, got)
         times[k], outs[k] = e0.elapsed_time(e1) / n_iter, got
     assert all(torch.equal(a, b) for a, b in zip(outs[0], outs[4]))
     # bound 0: about the mean of the maximum of four delays (320 us) per iteration
