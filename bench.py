@@ -61,6 +61,9 @@ def parse_args():
     ap.add_argument("--repeats", type=int, default=5,
                     help="repetitions of the timed loop at the headline bound for the mean and 95 %% confidence interval")
     ap.add_argument("--ks", default="", help="comma-separated bounds to time instead of the workload's own")
+    ap.add_argument("--ring", type=int, default=None, choices=[-1, 0, 1],
+                    help="persistent ring kernel: -1 only with injected delays, 0 also for small iterations, 1 always "
+                         "(default: the library's own choice)")
     return ap.parse_args()
 
 
@@ -303,6 +306,11 @@ def device_tables(w, bls, torch):
     return tabs
 
 
+def plan_iterations(bls, plan) -> int:
+    """Iterations the plan has issued so far (all ranks agree between loops)."""
+    return int(bls.bls_counters(plan)[0][0])
+
+
 def select(w, args):
     """Optional reductions of the workload for profiling runs."""
     import dataclasses
@@ -342,6 +350,8 @@ def run_mine(args):
 
     if args.tune:
         bls.bls_set_tuning(plan, *[int(x) for x in args.tune.split(",")])
+    if args.ring is not None:
+        bls.bls_set_ring(plan, args.ring)
     hot_k = HOT_DEFAULT.get(args.config, 0) if args.hot < 0 else args.hot
     if hot_k and w.partition == "table_rr":
         # request statistics come from two batches that are not among the timed ones
@@ -460,18 +470,45 @@ def run_mine(args):
                "d2h_bytes_per_step": int(h_out.numel() * 4), "steps": n_e2e, "k": k_head}
     delay_sweep = None
     if args.delay_us > 0:
-        # the paper's random-delay setting: bound 0 pays the largest delay every iteration, k > 0 hides part of it
-        delay_sweep = {}
+        # the paper's random-delay setting: bound 0 pays the largest delay every iteration, k > 0 hides the
+        # difference between the largest and the mean delay.  Beside each measured time: the oracle's timing
+        # recursion of Listing 2 for the same delays (reproduced on the host from the counter-based draw), and
+        # the paper's per-rank latency L = mean time between a rank's consecutive completions and throughput
+        # T = sum over ranks of batches / L (Section V-C), from the device's time stamps.
+        from oracle.ring_model import makespan       # the timing model is test infrastructure: reported beside, never used
+        span_ns, seed = int(2 * args.delay_us * 1000), 2024
+        n_d = min(args.steps, 1000)
+        rr = np.arange(w.P, dtype=np.uint64).reshape(-1, 1)
+        jj = np.arange(n_d, dtype=np.uint64).reshape(1, -1)
+        with np.errstate(over="ignore"):
+            z = np.uint64(seed) + ((rr << np.uint64(40)) + jj + np.uint64(1)) * np.uint64(0x9E3779B97F4A7C15)
+            z = (z ^ (z >> np.uint64(30))) * np.uint64(0xBF58476D1CE4E5B9)
+            z = (z ^ (z >> np.uint64(27))) * np.uint64(0x94D049BB133111EB)
+            z = z ^ (z >> np.uint64(31))
+        delays_us = (z % np.uint64(span_ns + 1)).astype(np.float64) / 1e3
+        # stall-free time per step in the same mode (ring kernel), the model's per-iteration work
+        bls.bls_set_ring(plan, 1)
+        loop(0, 5)
+        work_us = timed(0, n_d) / n_d * 1e3
+        delay_sweep = {"mean_delay_us": args.delay_us, "steps": n_d, "work_us": work_us,
+                       "closed_form_k0_us": work_us + 2 * args.delay_us * w.P / (w.P + 1),
+                       "closed_form_k_inf_us": work_us + args.delay_us}
+        u_d = float(sum(Ls[t % nd] for t in range(n_d)))
         for r in range(w.P):
-            bls.bls_set_random_stall(plan, r, int(2 * args.delay_us * 1000), 2024)
-        bls.bls_set_waves_per_step(plan, w.P + 1)
+            bls.bls_set_random_stall(plan, r, span_ns, seed)
         for k in ks:
-            ms, _ = aggregate(timed(k, args.steps), units, world, dev)
-            delay_sweep[str(k)] = {"ms_per_step": ms / args.steps}
+            it0 = bls.bls_profile_read(plan)["kernels_total"]
+            first = plan_iterations(bls, plan)
+            ms, _ = aggregate(timed(k, n_d), u_d, world, dev)
+            post, serve, done = bls.bls_timeline(plan, first, n_d)
+            lat = np.diff(done.astype(np.int64), axis=0).mean(axis=0) / 1e3          # us per batch, per logical rank
+            delay_sweep[str(k)] = {"us_per_step": ms / n_d * 1e3,
+                                   "model_us_per_step": makespan(delays_us, k, work=work_us) / n_d,
+                                   "latency_us_per_rank": [float(x) for x in lat],
+                                   "throughput_batches_per_s": float(np.sum(1e6 / lat)),
+                                   "launches": bls.bls_profile_read(plan)["kernels_total"] - it0}
         for r in range(w.P):
-            bls.bls_set_random_stall(plan, r, 0, 2024)
-        delay_sweep["mean_delay_us"] = args.delay_us
-        delay_sweep["expected_k0_extra_us"] = 2 * args.delay_us * w.P / (w.P + 1)
+            bls.bls_set_random_stall(plan, r, 0, seed)
     straggler = None
     if args.straggler:
         # every rank is delayed by the stall-free step time before each iteration, the last rank by twice that:

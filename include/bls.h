@@ -164,7 +164,7 @@ bls_status_t bls_step_host(bls_plan_t *plan, int k, const int32_t *ids /*host*/,
 bls_status_t bls_drain_host(bls_plan_t *plan, float *host_out /*host*/, int64_t *out_iter /*host out*/);
 
 /* ---- inspection (bls_view, bls_counters, bls_status, bls_set_poison, bls_set_wait_limit,
- * bls_profile*, bls_set_tuning: debugging and measurement aids with no counterpart in the paper) ---- */
+ * bls_profile*, bls_set_tuning, bls_set_overlap, bls_set_ring: debugging and measurement aids with no counterpart in the paper) ---- */
 /* Device pointers of the slot that holds iteration `iter` (must still be in the ring). */
 bls_status_t bls_view(bls_plan_t *plan, int64_t iter, bls_route_view_t *view /*host out*/);
 /* Synchronises the stream; copies the P per-rank counters to host arrays (may be NULL). */
@@ -174,22 +174,42 @@ bls_status_t bls_counters(bls_plan_t *plan, int64_t *posted, int64_t *served, in
  * posted iteration and the oldest incomplete one. */
 bls_status_t bls_status(bls_plan_t *plan, int64_t *max_lag /*host out*/);
 /* Injected delay of rank `rank` before each of its iterations (Section V-E,
- * setting 2: a delay models a slowdown of any nature), in nanoseconds. */
+ * setting 2: a delay models a slowdown of any nature), in nanoseconds.  As in Listing 2's
+ * loop the delay of iteration j + 1 starts when the rank has posted iteration j and has
+ * at most k requests outstanding; the rank posts iteration j + 1 when the delay is over.
+ * From the first injected delay on, the plan works with the persistent ring kernel (bls_set_ring). */
 bls_status_t bls_set_stall(bls_plan_t *plan, int rank, int64_t ns);
 /* The paper's random-delay setting: in addition to the fixed delay, rank `rank` is
  * delayed before each of its iterations by a time drawn uniformly from [0, max_ns]
  * (a counter-based draw from `seed`, the rank and the iteration number, so a run
  * can be repeated).  The seed is shared by all ranks of the plan. */
 bls_status_t bls_set_random_stall(bls_plan_t *plan, int rank, int64_t max_ns, uint64_t seed);
-/* While delays are injected, one bls_step runs up to `waves` waves of kernels (default 4,
- * at most P+1): while the iteration to hand back is still incomplete, a wave waits for the
- * earliest rank that can act (not for all of them), so ranks act at different moments and
- * faster ones run ahead; once it is complete waves do not wait; the last wave enforces the bound. */
-bls_status_t bls_set_waves_per_step(bls_plan_t *plan, int waves);
+/* The persistent ring kernel.  While delays are injected, every bls_step / bls_drain call is
+ * ONE cooperative kernel launch in which each logical rank runs the loop of Listing 2 on its own
+ * (Section III-C: initiation never synchronises two ranks): it spends its delay, completes the
+ * requests that have arrived, posts as soon as the slot of its next iteration is free (every
+ * rank has completed the iteration k + 1 before it), and blocks on its oldest request only while
+ * more than k are outstanding; owners answer an iteration as soon as all ranks have posted it.
+ * A scheduler warp publishes this work to the other blocks of the launch through a queue in the
+ * workspace; the launch ends once the call's iteration (t - k, or the drained one) is complete
+ * on every rank and nothing else can be done at that moment.  Results are the same bit for bit.
+ * mode -1 (default): only while delays are injected; 0: also for iterations below about 128 K
+ * lookups (one launch instead of three dependent ones), unless bls_set_overlap(1) was asked for;
+ * 1: always.  Only between loops (nothing outstanding), else BLS_ESTATE. */
+bls_status_t bls_set_ring(bls_plan_t *plan, int mode);
+/* Time stamps (device clock, ns) of the last 1024 iterations, for the per-rank latency and
+ * throughput the paper reports (Section V-C): for iterations first_iter .. first_iter + n_iter - 1
+ * and every rank r, when r's post of the iteration was complete, when owner r had answered it,
+ * and when r completed it.  Host arrays of n_iter * P entries indexed [i * P + r], any may be
+ * NULL.  Synchronises the stream.  BLS_ESTATE if an iteration has not been issued yet or is more
+ * than 1024 iterations old. */
+bls_status_t bls_timeline(bls_plan_t *plan, int64_t first_iter, int n_iter, uint64_t *post_ns /*host out*/,
+                          uint64_t *serve_ns /*host out*/, uint64_t *done_ns /*host out*/);
 /* Overlapped mode of bls_step (see there): mode 0 (default) uses it for iterations of about a
  * million lookups or more (P * max_ids_per_rank >= 2^20; smaller ones are bound by the launch
  * rate and lose to the second stream's extra driver calls), 1 whenever it applies (bound >= 1,
- * table-wise placement, no injected delays, no hot-row staging), -1 never.  May be called at any time. */
+ * table-wise placement, no injected delays, no hot-row staging, ring kernel not in use), -1 never.
+ * May be called at any time. */
 bls_status_t bls_set_overlap(bls_plan_t *plan, int mode);
 /* Debug aid: while enabled, the output slot an iteration is issued into is first filled
  * with 0xFF bytes (NaN), so that a bag that was not written, or a slot read before its data

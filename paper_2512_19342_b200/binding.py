@@ -25,7 +25,7 @@ EXPORTS = ["bls_plan_bytes", "bls_plan", "bls_destroy", "bls_route", "bls_lookup
            "bls_drain", "bls_step_host", "bls_drain_host", "bls_view", "bls_counters", "bls_status",
            "bls_set_stall", "bls_set_wait_limit", "bls_strerror", "bls_fill_hash_table",
            "bls_profile", "bls_profile_read", "bls_set_tuning", "bls_route_table_rr_static",
-           "bls_set_random_stall", "bls_set_waves_per_step", "bls_set_poison", "bls_set_overlap", "bls_a2a_bytes", "bls_a2a_create", "bls_a2a_destroy", "bls_a2a_post", "bls_a2a_wait",
+           "bls_set_random_stall", "bls_set_ring", "bls_timeline", "bls_set_poison", "bls_set_overlap", "bls_a2a_bytes", "bls_a2a_create", "bls_a2a_destroy", "bls_a2a_post", "bls_a2a_wait",
            "bls_a2a_status", "bls_hot_bytes", "bls_hot_attach", "bls_hot_observe", "bls_hot_build", "bls_hot_view"]
 
 
@@ -213,8 +213,18 @@ def bls_set_random_stall(plan: Plan, rank: int, max_ns: int, seed: int = 0) -> N
     _check(lib().bls_set_random_stall(plan.handle, rank, C.c_int64(max_ns), C.c_uint64(seed)), "bls_set_random_stall")
 
 
-def bls_set_waves_per_step(plan: Plan, waves: int) -> None:
-    _check(lib().bls_set_waves_per_step(plan.handle, waves), "bls_set_waves_per_step")
+def bls_set_ring(plan: Plan, mode: int) -> None:
+    """-1 persistent ring kernel only while delays are injected (default), 0 also for small iterations, 1 always."""
+    _check(lib().bls_set_ring(plan.handle, int(mode)), "bls_set_ring")
+
+
+def bls_timeline(plan: Plan, first_iter: int, n_iter: int):
+    """(post_ns, serve_ns, done_ns): three numpy uint64 arrays [n_iter][P] of device time stamps."""
+    import numpy as np
+    arrs = [np.zeros((n_iter, plan.P), np.uint64) for _ in range(3)]
+    _check(lib().bls_timeline(plan.handle, C.c_int64(first_iter), n_iter,
+                              *[a.ctypes.data_as(C.c_void_p) for a in arrs]), "bls_timeline")
+    return tuple(arrs)
 
 
 def bls_set_poison(plan: Plan, enable: bool) -> None:

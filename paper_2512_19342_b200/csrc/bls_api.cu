@@ -11,8 +11,8 @@ namespace {
 size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 struct Layout {
-    size_t dev, tab, pair, pair_of, pair_first, counts, sendbuf, sub_start, out, chunk_base, tile_cnt, rw_total, stage_ids,
-        stage_off, total;
+    size_t dev, tab, pair, pair_of, pair_first, counts, sendbuf, sub_start, out, chunk_base, tile_cnt, rw_total, queue,
+        stamps, stage_ids, stage_off, total;
 };
 
 int dtype_bytes(int dt) { return dt == BLS_F32 ? 4 : 2; }
@@ -90,6 +90,8 @@ Layout make_layout(const BlsParams &p)
     L.chunk_base = take(sizeof(int) * P * (size_t)(p.NI + 1));
     L.tile_cnt = take(p.part == BLS_PART_ROW_BLOCK ? sizeof(int) * P * (size_t)p.NT * P : 0);
     L.rw_total = take(p.part == BLS_PART_ROW_BLOCK ? sizeof(int) * P * P : 0);
+    L.queue = take(sizeof(BlsQueue));
+    L.stamps = take(sizeof(unsigned long long) * BLS_TL_ITERS * P * 3);
     L.stage_ids = take(sizeof(int) * S * P * (size_t)p.cap);
     L.stage_off = take(sizeof(int) * S * ((size_t)P * p.T * p.b + 1));
     L.total = o;
@@ -156,6 +158,8 @@ bls_status_t bls_plan(const bls_table_t *tables, int T, int part, int P, int loc
     p.chunk_base = (int *)(ws + L.chunk_base);
     p.tile_cnt = (int *)(ws + L.tile_cnt);
     p.rw_total = (int *)(ws + L.rw_total);
+    p.queue = (BlsQueue *)(ws + L.queue);
+    p.stamps = (unsigned long long *)(ws + L.stamps);
     p.stage_ids = (int *)(ws + L.stage_ids);
     p.stage_off = (int *)(ws + L.stage_off);
     pl->stream = (cudaStream_t)cuda_stream;
@@ -174,7 +178,7 @@ bls_status_t bls_plan(const bls_table_t *tables, int T, int part, int P, int loc
         int R = (int)((tw ? 160.0 : 50.0) / (avg < 0.5 ? 0.5 : avg) + 0.5);
         pl->bags_per_run = R < 4 ? 4 : (R > 24 ? 24 : R);
         pl->rows_in_flight = 4;
-        pl->max_waves = 4;
+        pl->ring_mode = -1;
     }
     int devid = 0;
     if (!cuda_ok(cudaGetDevice(&devid)) ||
@@ -233,6 +237,8 @@ bls_status_t bls_plan(const bls_table_t *tables, int T, int part, int P, int loc
               cuda_ok(cudaMemcpyAsync(ws + L.pair_first, pair_first.data(), sizeof(int) * (P + 1),
                                       cudaMemcpyHostToDevice, pl->stream)) &&
               cuda_ok(cudaMemsetAsync(ws + L.counts, 0, sizeof(int) * p.S * 4 * P * P, pl->stream)) &&
+              cuda_ok(cudaMemsetAsync(ws + L.queue, 0, 16, pl->stream)) &&            // the queue's header
+              cuda_ok(cudaMemsetAsync(ws + L.stamps, 0, sizeof(unsigned long long) * BLS_TL_ITERS * P * 3, pl->stream)) &&
               // the vectors above are pageable: make sure the copies have left them
               cuda_ok(cudaStreamSynchronize(pl->stream));
     if (!ok) { free(pl->h_rows); free(pl); return BLS_ECUDA; }
@@ -306,12 +312,12 @@ static bls_status_t launch_check()
 
 // One wave: gate -> router -> gather/pool/return -> commit, with optional stage events.
 static void enqueue_wave(bls_plan_t *pl, int mode, long long t_last, long long floor_, int k,
-                         const int *ids, const int *off, long long n_ids, int opportunistic = 0)
+                         const int *ids, const int *off, long long n_ids)
 {
     cudaEvent_t *ev = nullptr;
     if (pl->prof_on && pl->prof_n < BLS_PROF_MAX && pl->prof_ev) ev = pl->prof_ev + (size_t)pl->prof_n++ * 4;
     if (ev) cudaEventRecord(ev[0], pl->stream);
-    bls_launch_gate(pl, mode, t_last, floor_, k, ids, off, n_ids, opportunistic);
+    bls_launch_gate(pl, mode, t_last, floor_, k, ids, off, n_ids);
     bls_launch_route(pl);
     if (ev) cudaEventRecord(ev[1], pl->stream);
     bls_launch_gather(pl);                             // its last block commits the wave
@@ -347,7 +353,7 @@ static void enqueue_wave_overlapped(bls_plan_t *pl, long long t_last, long long 
     cudaEvent_t *ev = nullptr;
     if (pl->prof_on && pl->prof_n < BLS_PROF_MAX && pl->prof_ev) ev = pl->prof_ev + (size_t)pl->prof_n++ * 4;
     if (ev) cudaEventRecord(ev[0], pl->stream);
-    bls_launch_gate(pl, BLS_MODE_STEP, t_last, floor_, k, ids, off, n_ids, 0, 1);
+    bls_launch_gate(pl, BLS_MODE_STEP, t_last, floor_, k, ids, off, n_ids, 1);
     cudaEventRecord(pl->e_fork, pl->stream);
     if (ev) cudaEventRecord(ev[1], pl->stream);
     bls_launch_gather(pl);                             // first, so that its blocks are resident first
@@ -358,6 +364,33 @@ static void enqueue_wave_overlapped(bls_plan_t *pl, long long t_last, long long 
     cudaStreamWaitEvent(pl->stream, pl->e_join, 0);
     if (ev) { cudaEventRecord(ev[2], pl->stream); cudaEventRecord(ev[3], pl->stream); }
     pl->kernels_launched += 3 + bls_route_kernels(pl);
+}
+
+// Event-driven mode: the whole call is one launch of the persistent ring kernel, in which
+// every logical rank posts, is answered and completes on its own (bls_event.cu).  Used
+// whenever delays are injected, and for iterations so small that the launches of a wave
+// would dominate.
+static bool ring_applies(const bls_plan_t *pl)
+{
+    if (pl->any_stall || pl->ring_mode > 0) return true;
+    // small iterations (below about 128 K lookups): one launch instead of three dependent ones,
+    // unless the caller asked for the overlapped mode of the stand-alone kernels
+    return pl->ring_mode == 0 && pl->overlap_mode <= 0 && !pl->prm.hot.enabled &&
+           (long long)pl->prm.P * pl->prm.cap < (1 << 17);
+}
+
+static bls_status_t enqueue_ring(bls_plan_t *pl, int mode, long long t_last, long long floor_, int k, const int *ids,
+                                 const int *off, long long n_ids)
+{
+    cudaEvent_t *ev = nullptr;
+    if (pl->prof_on && pl->prof_n < BLS_PROF_MAX && pl->prof_ev) ev = pl->prof_ev + (size_t)pl->prof_n++ * 4;
+    if (ev) { cudaEventRecord(ev[0], pl->stream); cudaEventRecord(ev[1], pl->stream); }
+    const int err = bls_launch_ring(pl, mode, t_last, floor_, k, ids, off, n_ids);
+    if (ev) { cudaEventRecord(ev[2], pl->stream); cudaEventRecord(ev[3], pl->stream); }
+    pl->kernels_launched += 1;
+    pl->unserved = 0;                                  // whatever the owners still owe is answered inside the launch
+    pl->ring_used = 1;
+    return err == (int)cudaSuccess ? BLS_OK : BLS_ECUDA;
 }
 
 // Debug aid: a slot that is about to receive iteration `iter` holds an iteration that has
@@ -381,7 +414,7 @@ bls_status_t bls_route(bls_plan_t *pl, int64_t iter, const int32_t *ids, const i
     if (!pl || !offsets || (!ids && n_ids > 0) || n_ids < 0) return BLS_EINVAL;
     if (iter != pl->t_next || pl->t_handed != pl->t_next || pl->routed_only >= 0) return BLS_ESTATE;
     poison_slot(pl, iter);
-    bls_launch_gate(pl, BLS_MODE_ROUTE_ONLY, iter, -1, 0, ids, offsets, n_ids, 0);
+    bls_launch_gate(pl, BLS_MODE_ROUTE_ONLY, iter, -1, 0, ids, offsets, n_ids);
     bls_launch_route(pl);
     bls_launch_commit(pl);
     pl->kernels_launched += 2 + bls_route_kernels(pl);
@@ -394,7 +427,7 @@ bls_status_t bls_lookup(bls_plan_t *pl, int64_t iter)
 {
     if (!pl) return BLS_EINVAL;
     if (pl->routed_only != iter) return BLS_ESTATE;
-    bls_launch_gate(pl, BLS_MODE_LOOKUP_ONLY, iter, -1, 0, nullptr, nullptr, 0, 0);
+    bls_launch_gate(pl, BLS_MODE_LOOKUP_ONLY, iter, -1, 0, nullptr, nullptr, 0);
     bls_launch_gather(pl);                             // its last block commits the wave
     pl->kernels_launched += 2;
     pl->routed_only = -1;
@@ -411,22 +444,20 @@ bls_status_t bls_step(bls_plan_t *pl, int k, const int32_t *ids, const int32_t *
     pl->k_cur = k;
     const long long t = pl->t_next++;
     poison_slot(pl, t);
-    // With injected delays the ranks act at different moments: a few opportunistic waves
-    // (while the iteration to hand back is incomplete they wait for the earliest rank that can act) let them drift apart and catch
-    // up, the last wave enforces the bound.  Without delays one wave does everything.
-    const int waves = pl->any_stall ? (pl->max_waves < pl->prm.P + 1 ? pl->max_waves : pl->prm.P + 1) : 1;
     // (iterations below about a million lookups are bound by the launch rate, of the host or of
     // the GPU, and the second stream costs five more driver calls per step: they stay on one stream)
-    const bool overlapped = k >= 1 && !pl->any_stall && pl->prm.part == BLS_PART_TABLE_RR && !pl->prm.hot.enabled &&
+    const bool ring = ring_applies(pl);
+    const bool overlapped = !ring && k >= 1 && pl->prm.part == BLS_PART_TABLE_RR && !pl->prm.hot.enabled &&
                             pl->overlap_mode >= 0 &&
                             (pl->overlap_mode > 0 || (long long)pl->prm.P * pl->prm.cap >= (1 << 20)) && side_stream_ready(pl);
-    if (overlapped) {
+    if (ring) {
+        const bls_status_t st = enqueue_ring(pl, BLS_MODE_STEP, t, t - k, k, ids, offsets, n_ids);
+        if (st != BLS_OK) return st;
+    } else if (overlapped) {
         enqueue_wave_overlapped(pl, t, t - k, k, ids, offsets, n_ids);
         pl->unserved = 1;                              // iteration t is answered by the next wave
     } else {
-        for (int v = 0; v + 1 < waves; v++)
-            enqueue_wave(pl, BLS_MODE_STEP, t, t - k, k, ids, v == 0 ? offsets : nullptr, n_ids, 1);
-        enqueue_wave(pl, BLS_MODE_STEP, t, t - k, k, ids, waves == 1 ? offsets : nullptr, n_ids);
+        enqueue_wave(pl, BLS_MODE_STEP, t, t - k, k, ids, offsets, n_ids);
     }
     if (t - k >= 0) {
         *out = slot_out(pl, t - k);
@@ -447,20 +478,24 @@ bls_status_t bls_drain(bls_plan_t *pl, const float **out, int64_t *out_iter)
         *out = nullptr;
         *out_iter = -1;
         pl->k_cur = -1;
+        pl->ring_used = 0;
         return BLS_OK;
     }
     const long long f = pl->t_handed;
-    // Without injected delays every rank completes an iteration in the step that issues
-    // it (in overlapped mode: in the step after it, so the newest one is still to be
-    // answered); otherwise the outstanding iterations are already complete on the stream.
-    if (pl->any_stall || pl->unserved) {
+    // In a wave every rank completes an iteration in the step that issues it (in overlapped
+    // mode: in the step after it, so the newest one is still to be answered).  In event-driven
+    // mode ranks may be behind: the launch ends once iteration f is complete on every rank.
+    if (pl->any_stall || pl->ring_used) {
+        const bls_status_t st = enqueue_ring(pl, BLS_MODE_DRAIN, pl->t_next - 1, f, pl->k_cur < 0 ? 0 : pl->k_cur, nullptr, nullptr, 0);
+        if (st != BLS_OK) return st;
+    } else if (pl->unserved) {
         enqueue_wave(pl, BLS_MODE_DRAIN, pl->t_next - 1, f, pl->k_cur < 0 ? 0 : pl->k_cur, nullptr, nullptr, 0);
         pl->unserved = 0;
     }
     *out = slot_out(pl, f);
     *out_iter = f;
     pl->t_handed = f + 1;
-    if (pl->t_handed == pl->t_next) pl->k_cur = -1;
+    if (pl->t_handed == pl->t_next) { pl->k_cur = -1; pl->ring_used = 0; }
     return launch_check();
 }
 
@@ -624,10 +659,31 @@ bls_status_t bls_set_overlap(bls_plan_t *pl, int mode)
     return BLS_OK;
 }
 
-bls_status_t bls_set_waves_per_step(bls_plan_t *pl, int waves)
+bls_status_t bls_set_ring(bls_plan_t *pl, int mode)
 {
-    if (!pl || waves < 1 || waves > 64) return BLS_EINVAL;
-    pl->max_waves = waves;
+    if (!pl || mode < -1 || mode > 1) return BLS_EINVAL;
+    if (pl->t_handed != pl->t_next) return BLS_ESTATE;      // only between loops
+    pl->ring_mode = mode;
+    return BLS_OK;
+}
+
+bls_status_t bls_timeline(bls_plan_t *pl, int64_t first_iter, int n_iter, uint64_t *post_ns, uint64_t *serve_ns,
+                          uint64_t *done_ns)
+{
+    if (!pl || first_iter < 0 || n_iter < 0) return BLS_EINVAL;
+    if (first_iter + n_iter > pl->t_next || first_iter + BLS_TL_ITERS < pl->t_next) return BLS_ESTATE;
+    if (cudaStreamSynchronize(pl->stream) != cudaSuccess) return BLS_ECUDA;
+    const int P = pl->prm.P;
+    std::vector<unsigned long long> h((size_t)BLS_TL_ITERS * P * 3);
+    if (cudaMemcpy(h.data(), pl->prm.stamps, h.size() * sizeof(unsigned long long), cudaMemcpyDeviceToHost) != cudaSuccess)
+        return BLS_ECUDA;
+    for (int i = 0; i < n_iter; i++)
+        for (int r = 0; r < P; r++) {
+            const unsigned long long *e = &h[((size_t)((first_iter + i) % BLS_TL_ITERS) * P + r) * 3];
+            if (post_ns) post_ns[(size_t)i * P + r] = e[0];
+            if (serve_ns) serve_ns[(size_t)i * P + r] = e[1];
+            if (done_ns) done_ns[(size_t)i * P + r] = e[2];
+        }
     return BLS_OK;
 }
 

@@ -12,6 +12,62 @@ __device__ __forceinline__ unsigned long long globaltimer_ns()
 
 __device__ __forceinline__ void flag(const BlsParams &p, int bit) { atomicOr(&p.dev->status, bit); }
 
+// Injected delay of rank r before it posts iteration j: the fixed part plus a uniform draw
+// from [0, span], the SplitMix64 output for (seed, rank, iteration) - a counter-based
+// generator, so a run can be repeated and reproduced on the host.
+__device__ __forceinline__ unsigned long long stall_draw(const BlsDev *d, int r, long long j)
+{
+    unsigned long long stall = d->stall_ns[r];
+    const unsigned long long span = d->stall_rand_ns[r];
+    if (span) {
+        unsigned long long z = d->stall_seed + (((unsigned long long)r << 40) + (unsigned long long)j + 1ull) * 0x9E3779B97F4A7C15ull;
+        z = (z ^ (z >> 30)) * 0xBF58476D1CE4E5B9ull;
+        z = (z ^ (z >> 27)) * 0x94D049BB133111EBull;
+        z ^= z >> 31;
+        stall += z % (span + 1ull);
+    }
+    return stall;
+}
+
+// Time stamp of an event of (iteration j, rank r): what = 0 post, 1 serve, 2 completion.
+__device__ __forceinline__ void stamp(const BlsParams &p, long long j, int r, int what, unsigned long long now)
+{
+    p.stamps[((size_t)(j % BLS_TL_ITERS) * p.P + r) * 3 + what] = now;
+}
+
+// Receive-side counts and displacements of the request leg for owner r, iteration j
+// (recvcounts = sendcounts transposed, rdispls = exclusive scan over sources).
+__device__ __forceinline__ void write_recv_side(const BlsParams &p, int r, long long j)
+{
+    int *cnt = p.counts + (size_t)(j % p.S) * 4 * p.P * p.P;
+    const int *sendcounts = cnt;
+    int *recvcounts = cnt + 2 * p.P * p.P, *rdispls = cnt + 3 * p.P * p.P;
+    int run = 0;
+    for (int src = 0; src < p.P; src++) {
+        const int c = sendcounts[src * p.P + r];
+        recvcounts[r * p.P + src] = c;
+        rdispls[r * p.P + src] = run;
+        run += c;
+    }
+}
+
+__device__ __forceinline__ long long warp_min_ll(long long v)
+{
+    for (int o = 16; o > 0; o >>= 1) {
+        long long w = __shfl_xor_sync(0xffffffffu, v, o);
+        v = w < v ? w : v;
+    }
+    return v;
+}
+__device__ __forceinline__ long long warp_max_ll(long long v)
+{
+    for (int o = 16; o > 0; o >>= 1) {
+        long long w = __shfl_xor_sync(0xffffffffu, v, o);
+        v = w > v ? w : v;
+    }
+    return v;
+}
+
 // What a requester needs to route the iteration the gate assigned to it.
 struct RouteCtx {
     const int *ids, *off;
@@ -90,10 +146,8 @@ __device__ __forceinline__ void tw_meta_warp(const BlsParams &p, int src, int la
     }
 }
 
-// Publish the progress of the wave that has just run (lane r = rank r) and start the
-// injected delay of every rank that posted.  For every answered iteration also write
-// the receive-side counts and displacements of the request leg (recvcounts =
-// sendcounts transposed, rdispls = exclusive scan over sources).
+// Publish the progress of the wave that has just run (lane r = rank r).  For every
+// answered iteration also write the receive-side counts and displacements.
 __device__ __forceinline__ void commit_lane(const BlsParams &p, int r)
 {
     BlsDev *d = p.dev;
@@ -102,39 +156,22 @@ __device__ __forceinline__ void commit_lane(const BlsParams &p, int r)
     long long j = d->route_iter[r];
     if (j >= 0) {
         d->posted[r] = j + 1;
-        unsigned long long stall = d->stall_ns[r];
-        const unsigned long long span = d->stall_rand_ns[r];
-        if (span) {
-            // uniform in [0, span]: SplitMix64 output for (seed, rank, iteration), a counter-based draw
-            unsigned long long z = d->stall_seed + (((unsigned long long)r << 40) + (unsigned long long)j + 1ull) * 0x9E3779B97F4A7C15ull;
-            z = (z ^ (z >> 30)) * 0xBF58476D1CE4E5B9ull;
-            z = (z ^ (z >> 27)) * 0x94D049BB133111EBull;
-            z ^= z >> 31;
-            stall += z % (span + 1ull);
-        }
-        d->ready_ns[r] = now + stall;
+        stamp(p, j, r, 0, now);
         // route_iter stays as it is until the next gate rewrites it: in overlapped mode the
         // router of this wave may still be running beside the kernel that commits
     }
     j = d->serve_iter[r];
     if (j >= 0) {
-        int *cnt = p.counts + (size_t)(j % p.S) * 4 * p.P * p.P;
-        const int *sendcounts = cnt;
-        int *recvcounts = cnt + 2 * p.P * p.P, *rdispls = cnt + 3 * p.P * p.P;
-        int run = 0;
-        for (int src = 0; src < p.P; src++) {
-            int c = sendcounts[src * p.P + r];
-            recvcounts[r * p.P + src] = c;
-            rdispls[r * p.P + src] = run;
-            run += c;
-        }
+        write_recv_side(p, r, j);
         d->served[r] = j + 1;
         d->serve_iter[r] = -1;
+        stamp(p, j, r, 1, now);
     }
     j = d->consume_iter[r];
     if (j >= 0) {
         d->done[r] = j + 1;
         d->consume_iter[r] = -1;
+        stamp(p, j, r, 2, now);
     }
 }
 

@@ -14,6 +14,36 @@ enum { BLS_MODE_STEP = 0, BLS_MODE_DRAIN = 1, BLS_MODE_ROUTE_ONLY = 2, BLS_MODE_
 // bits of the device status word
 enum { BLS_ST_EINVAL = 1, BLS_ST_ENOSPC = 2, BLS_ST_ERANGE = 4, BLS_ST_ETIMEOUT = 8, BLS_ST_ESTATE = 16 };
 
+// ---- persistent ring kernel (bls_event.cu): a queue of actions that a scheduler warp
+// publishes and worker blocks execute tile by tile, all inside one launch ----
+#define BLS_Q_CAP 4096            // actions one launch can publish: at most (k_max + 1) iterations x 4 P
+enum { BLS_ACT_TW_META = 0, BLS_ACT_TW_COPY, BLS_ACT_RW_COUNT, BLS_ACT_RW_SCAN, BLS_ACT_RW_SCATTER,
+       BLS_ACT_GATHER_TW, BLS_ACT_GATHER_RW };
+struct BlsAct {
+    int kind;           // BLS_ACT_*
+    int rank;           // requester (router actions) or owner (table-wise gather)
+    int slot;           // ring slot of the iteration
+    int n_tiles;        // tiles of BLS_ROUTE_TB threads' work
+    int next;           // next tile to hand out (atomic)
+    int finished;       // tiles completed (atomic)
+    int aux;            // gather actions: number of runs
+    int first;          // table-wise gather: the owner's first (owner, table) pair
+};
+struct BlsQueue {
+    unsigned tail;      // actions published so far in this launch (release / acquire)
+    int exit;           // set by the scheduler when the launch is over
+    int exited;         // blocks that have left; the last one clears this header for the next launch
+    int pad;
+    BlsAct act[BLS_Q_CAP];
+};
+// what a logical rank is doing between two posts (event-driven mode)
+enum { BLS_RS_IDLE = 0,        // previous iteration dealt with; the delay of the next one has not started
+       BLS_RS_DELAY = 1,       // inside its injected delay (until ready_ns)
+       BLS_RS_WANT_POST = 2,   // ready to post as soon as the slot is free and the inputs are there
+       BLS_RS_POSTING = 3,     // router actions in flight
+       BLS_RS_AFTER_POST = 4 };// posted; completes what has arrived, blocks while more than k are outstanding
+#define BLS_TL_ITERS 1024         // iterations whose time stamps are kept (a ring indexed by iteration mod this)
+
 // Device-resident state of the slot ring.  Counters are monotone: posted[r] =
 // iterations whose requests rank r has put into the owners' slots, served[o] =
 // iterations owner o has answered, done[r] = iterations rank r has completed.
@@ -33,6 +63,7 @@ struct BlsDev {
     const int *in_ids[BLS_MAX_SLOTS];
     const int *in_off[BLS_MAX_SLOTS];
     long long in_n[BLS_MAX_SLOTS];
+    int rstate[BLS_MAX_RANKS];                    // BLS_RS_*: event-driven mode only
     unsigned long long wait_limit_ns;
     long long max_lag;                            // max over time of newest posted - oldest incomplete
     int status;                                   // OR of BLS_ST_* bits
@@ -96,6 +127,8 @@ struct BlsParams {
     int *chunk_base;             // [P][NI+1]   table-wise: start of each (src, table) chunk
     int *tile_cnt;               // [P][NT][P]  row-wise: per tile, per destination counts / bases
     int *rw_total;               // [P][P]      row-wise: lookups of requester src that go to d (zeroed by the gate)
+    BlsQueue *queue;             // action queue of the persistent ring kernel
+    unsigned long long *stamps;  // [BLS_TL_ITERS][P][3] globaltimer at post / serve / completion of (iteration, rank)
     int *stage_ids;              // [S][P*cap]  staging for host inputs
     int *stage_off;              // [S][G+1]
     long long sub_stride;        // NQ + 1 rounded up to a multiple of 4
@@ -126,7 +159,9 @@ struct bls_plan {
     int bags_per_run;             // gather kernel: consecutive sub-bags streamed by one lane group
     int rows_in_flight;           // gather kernel: row loads per batch (4 or 8)
     long long *h_rows;            // host copy of the table heights
-    int max_waves;                // with injected delays: waves per step (the last one enforces the bound)
+    int ring_used;                // the loop in progress has used the ring kernel: its drain does too (ranks may be behind)
+    int ring_mode;                // persistent ring kernel: -1 only with injected delays, 0 also for small iterations, 1 always
+    int ring_blocks_per_sm;       // resident blocks of the ring kernel per SM (0 = not queried yet)
     int poison;                   // debug: fill an output slot with NaN patterns before an iteration is issued into it
     int hot_attached;             // a hot-row buffer has been attached
     // overlapped mode (bound >= 1, table-wise, no injected delays): the router of iteration t
@@ -141,7 +176,11 @@ struct bls_plan {
 
 // kernel launchers (defined in the .cu files)
 void bls_launch_gate(const bls_plan_t *pl, int mode, long long t_last, long long forced_floor, int k,
-                     const int *ids, const int *off, long long n_ids, int opportunistic, int overlapped = 0);
+                     const int *ids, const int *off, long long n_ids, int overlapped = 0);
+// one launch of the persistent ring kernel (event-driven mode); returns a cudaError_t as int
+int bls_launch_ring(bls_plan_t *pl, int mode, long long t_last, long long floor_, int k,
+                    const int *ids, const int *off, long long n_ids);
+void bls_gather_tiling(const bls_plan_t *pl, int *R, int *runs_per_chunk);   // run length the gather kernels use
 void bls_launch_commit(const bls_plan_t *pl);
 void bls_launch_meta(const bls_plan_t *pl, cudaStream_t stream);   // table-wise router, first half, as a kernel of its own
 void bls_launch_route(const bls_plan_t *pl);

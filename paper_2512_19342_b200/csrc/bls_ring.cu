@@ -12,33 +12,18 @@
 //   * a rank completes iteration j once all owners have answered it; completion
 //     is oldest first; the oldest request must complete once more than k are
 //     outstanding; the last batch drains everything.
-// A rank under an injected delay takes no action until its delay has passed,
-// unless the bound forces it; then the gate waits (bounded) on the clock.
+// Without injected delays all ranks act together, one wave of stand-alone kernels per
+// step, planned by the gate below.  With injected delays the ranks act on their own,
+// inside the persistent ring kernel of bls_event.cu, under the same rules.
 #include "bls_device.cuh"
-
-__device__ __forceinline__ long long warp_min_ll(long long v)
-{
-    for (int o = 16; o > 0; o >>= 1) {
-        long long w = __shfl_xor_sync(0xffffffffu, v, o);
-        v = w < v ? w : v;
-    }
-    return v;
-}
-__device__ __forceinline__ long long warp_max_ll(long long v)
-{
-    for (int o = 16; o > 0; o >>= 1) {
-        long long w = __shfl_xor_sync(0xffffffffu, v, o);
-        v = w > v ? w : v;
-    }
-    return v;
-}
 
 // Warp 0 decides (lane r is logical rank r).  With table-wise placement the block has
 // one more warp per rank, which then runs the first half of the router for the ranks
 // that were told to post (saves a launch on the critical path of every step).
+// This gate plans one wave of stand-alone kernels and never waits: injected delays are
+// the business of the event-driven ring kernel (bls_event.cu).
 __device__ __forceinline__ void gate_warp(const BlsParams &p, int mode, long long t_last, long long floor_, int k,
-                                          const int *ids, const int *off, long long n_ids, int opportunistic,
-                                          int overlapped)
+                                          const int *ids, const int *off, long long n_ids, int overlapped)
 {
     BlsDev *d = p.dev;
     const int r = threadIdx.x;
@@ -58,53 +43,14 @@ __device__ __forceinline__ void gate_warp(const BlsParams &p, int mode, long lon
     }
     __syncwarp();
 
-    long long posted = act ? d->posted[r] : BIG;
-    long long served = act ? d->served[r] : BIG;
-    long long done = act ? d->done[r] : BIG;
-    unsigned long long ready_at = act ? d->ready_ns[r] : 0ull;
+    const long long posted = act ? d->posted[r] : BIG;
+    const long long served = act ? d->served[r] : BIG;
+    const long long done = act ? d->done[r] : BIG;
     const bool sync_mode = (mode == BLS_MODE_ROUTE_ONLY || mode == BLS_MODE_LOOKUP_ONLY);
-
-    // Ranks the bound forces to act: anything still at or below the floor.  Only the last
-    // wave of a step forces them (and waits, bounded, for their injected delays).  An earlier
-    // wave waits only while the step's obligation - everything up to the floor complete - is
-    // unmet, and then only for the earliest rank that could act, so that faster ranks keep
-    // running ahead while a slow one is awaited; once the obligation is met it never waits.
-    const bool at_floor = act && floor_ >= 0 && (posted <= floor_ || served <= floor_ || done <= floor_);
-    const bool forced = act && (sync_mode || (!opportunistic && at_floor));
-    unsigned long long need = forced ? ready_at : 0ull;
-    for (int o = 16; o > 0; o >>= 1) {
-        unsigned long long w = __shfl_xor_sync(0xffffffffu, need, o);
-        need = w > need ? w : need;
-    }
-    unsigned long long now = globaltimer_ns();
-    if (opportunistic) {
-        need = 0ull;
-        if (__any_sync(0xffffffffu, at_floor)) {
-            const long long mp = warp_min_ll(posted), ms = warp_min_ll(served), md = warp_min_ll(done);
-            const bool could = act && ((posted <= t_last && md >= posted - k) || served < mp || done < ms);
-            unsigned long long first = could ? ready_at : ~0ull;
-            for (int o = 16; o > 0; o >>= 1) {
-                unsigned long long w = __shfl_xor_sync(0xffffffffu, first, o);
-                first = w < first ? w : first;
-            }
-            need = first == ~0ull ? 0ull : first;
-        }
-    }
-    if (!sync_mode && need > now) {
-        const unsigned long long give_up = now + d->wait_limit_ns;
-        while (now < need && now < give_up) {
-            __nanosleep(1000);
-            now = globaltimer_ns();
-        }
-        if (now < need && r == 0) atomicOr(&d->status, BLS_ST_ETIMEOUT);
-    }
-    const bool is_ready = forced || now >= ready_at;
-
     const long long min_done = warp_min_ll(done);
 
     // post: slot of iteration `posted` is free once every rank completed posted - k - 1
-    bool go_r = act && mode != BLS_MODE_LOOKUP_ONLY && posted <= t_last &&
-                min_done >= posted - k && is_ready;
+    bool go_r = act && mode != BLS_MODE_LOOKUP_ONLY && posted <= t_last && min_done >= posted - k;
     long long posted2 = act ? posted + (go_r ? 1 : 0) : BIG;
     const long long min_posted2 = warp_min_ll(posted2);
     const long long max_posted2 = warp_max_ll(act ? posted2 : -1);
@@ -113,18 +59,12 @@ __device__ __forceinline__ void gate_warp(const BlsParams &p, int mode, long lon
     // router of this wave runs beside the gather kernel, so only iterations posted by earlier
     // waves can be answered.
     const long long min_posted = warp_min_ll(posted);
-    bool go_s = act && mode != BLS_MODE_ROUTE_ONLY && served < (overlapped ? min_posted : min_posted2) && is_ready;
-    if (p.part == BLS_PART_ROW_BLOCK) {
-        // row-wise: a bag needs all owners' partial sums at once, so the owners answer an
-        // iteration together, when all of them are free to act
-        const bool all_ready = __all_sync(0xffffffffu, !act || is_ready);
-        go_s = go_s && all_ready;
-    }
+    bool go_s = act && mode != BLS_MODE_ROUTE_ONLY && served < (overlapped ? min_posted : min_posted2);
     long long served2 = act ? served + (go_s ? 1 : 0) : BIG;
     const long long min_served2 = warp_min_ll(served2);
 
     // complete: all owners have answered; oldest first
-    bool go_c = act && mode != BLS_MODE_ROUTE_ONLY && done < min_served2 && is_ready;
+    bool go_c = act && mode != BLS_MODE_ROUTE_ONLY && done < min_served2;
     long long done2 = act ? done + (go_c ? 1 : 0) : BIG;
     const long long min_done2 = warp_min_ll(done2);
 
@@ -137,7 +77,7 @@ __device__ __forceinline__ void gate_warp(const BlsParams &p, int mode, long lon
         long long lag = max_posted2 - 1 - min_done;
         if (lag > d->max_lag) d->max_lag = lag;
         // the wave must satisfy the bound: everything up to the floor completes
-        if (!sync_mode && !opportunistic && floor_ >= 0 && min_done2 <= floor_) atomicOr(&d->status, BLS_ST_ESTATE);
+        if (!sync_mode && floor_ >= 0 && min_done2 <= floor_) atomicOr(&d->status, BLS_ST_ESTATE);
         if (mode == BLS_MODE_ROUTE_ONLY && min_posted2 <= t_last) atomicOr(&d->status, BLS_ST_ESTATE);
         if (mode == BLS_MODE_LOOKUP_ONLY && min_done2 <= t_last) atomicOr(&d->status, BLS_ST_ESTATE);
     }
@@ -145,10 +85,9 @@ __device__ __forceinline__ void gate_warp(const BlsParams &p, int mode, long lon
 
 __global__ void __launch_bounds__(1024) bls_gate_kernel(BlsParams p, int mode, long long t_last,
                                                         long long floor_, int k, const int *ids,
-                                                        const int *off, long long n_ids, int opportunistic,
-                                                        int overlapped)
+                                                        const int *off, long long n_ids, int overlapped)
 {
-    if (threadIdx.x < 32) gate_warp(p, mode, t_last, floor_, k, ids, off, n_ids, opportunistic, overlapped);
+    if (threadIdx.x < 32) gate_warp(p, mode, t_last, floor_, k, ids, off, n_ids, overlapped);
     // overlapped mode: the router's first half runs on the second stream too (bls_tw_meta_kernel)
     if (p.part != BLS_PART_TABLE_RR || mode == BLS_MODE_LOOKUP_ONLY || overlapped) return;
     __threadfence_block();
@@ -174,11 +113,11 @@ void bls_launch_meta(const bls_plan_t *pl, cudaStream_t stream)
 __global__ void __launch_bounds__(32) bls_commit_kernel(BlsParams p) { commit_lane(p, threadIdx.x); }
 
 void bls_launch_gate(const bls_plan_t *pl, int mode, long long t_last, long long forced_floor, int k,
-                     const int *ids, const int *off, long long n_ids, int opportunistic, int overlapped)
+                     const int *ids, const int *off, long long n_ids, int overlapped)
 {
     // table-wise: one warp per rank for the router's first half (warp 0 is also the gate)
     const bool meta = pl->prm.part == BLS_PART_TABLE_RR && mode != BLS_MODE_LOOKUP_ONLY && !overlapped;
-    bls_gate_kernel<<<1, meta ? 32 * pl->prm.P : 32, 0, pl->stream>>>(pl->prm, mode, t_last, forced_floor, k, ids, off, n_ids, opportunistic, overlapped);
+    bls_gate_kernel<<<1, meta ? 32 * pl->prm.P : 32, 0, pl->stream>>>(pl->prm, mode, t_last, forced_floor, k, ids, off, n_ids, overlapped);
 }
 
 void bls_launch_commit(const bls_plan_t *pl)

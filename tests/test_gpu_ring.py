@@ -22,9 +22,13 @@ def assert_matches_oracle(w, data, inputs, outs):
         assert err <= TOL[w.tables[0].dtype], (it, err)
 
 
-def run_loop(w, tabs, k, n_iter, k_max=None, stalls=None, check_views=False, wait_limit=None):
-    """Listing 2's loop: n_iter steps then the drain; returns {iteration: output}."""
+def run_loop(w, tabs, k, n_iter, k_max=None, stalls=None, check_views=False, wait_limit=None, ring=None):
+    """Listing 2's loop: n_iter steps then the drain; returns {iteration: output}.
+    ring = 1 runs every call as one launch of the persistent ring kernel (which is also what
+    injected delays switch on); None leaves the plan's default (stand-alone kernels)."""
     plan = make_plan(w, tabs, k if k_max is None else k_max)
+    if ring is not None:
+        bls.bls_set_ring(plan, ring)
     if wait_limit is not None:
         bls.bls_set_wait_limit(plan, wait_limit)
     for r, ns in (stalls or {}).items():
@@ -58,20 +62,21 @@ def run_loop(w, tabs, k, n_iter, k_max=None, stalls=None, check_views=False, wai
     return outs, inputs, status, lag
 
 
-@pytest.mark.parametrize("num,rs,bs", [(1, 1.0, 1.0), (3, 0.01, 0.02), (4, 0.002, 0.01)])
-def test_output_is_independent_of_k(num, rs, bs):
+@pytest.mark.parametrize("ring", [None, 1], ids=["kernels", "ring"])
+@pytest.mark.parametrize("num,rs,bs", [(1, 1.0, 1.0), (3, 0.01, 0.02), (4, 0.002, 0.01), (5, 0.001, 0.003)])
+def test_output_is_independent_of_k(num, rs, bs, ring):
     w = bi.workload(num, rs, bs)
     data = [bi.table_values(t) for t in w.tables]
     tabs = dev_tables(w, data)
     n_iter = 7
-    ref, inputs, status, lag = run_loop(w, tabs, 0, n_iter, check_views=True)
+    ref, inputs, status, lag = run_loop(w, tabs, 0, n_iter, check_views=True, ring=ring)
     assert status == bls.BLS_OK and lag == 0 and sorted(ref) == list(range(n_iter))
     P, T, b = w.P, w.T, w.local_batch
     for it, (ids, off) in enumerate(inputs):
         want = oracle.pool_definition(P, T, b, w.tables, data, ids, off)
         assert oracle.vector_rel_err(ref[it].cpu().numpy(), want) <= TOL[w.tables[0].dtype]
     for k in (1, 2, 4, 8):
-        outs, _, status, lag = run_loop(w, tabs, k, n_iter, check_views=True)
+        outs, _, status, lag = run_loop(w, tabs, k, n_iter, check_views=True, ring=ring)
         assert status == bls.BLS_OK and lag <= k
         assert sorted(outs) == list(range(n_iter))
         for it in range(n_iter):
@@ -220,22 +225,121 @@ def test_host_buffer_entry_points():
         assert oracle.vector_rel_err(got[it].numpy(), want) <= 1e-5
 
 
-def test_random_delays_are_masked_by_the_bound():
-    """Section V-E setting 2 / Section VI-B: every rank is delayed by a uniform random time
-    before each iteration.  Bound 0 pays the largest of the P delays in every iteration;
-    a bound k > 0 lets ranks drift apart and hides part of it.  Results do not change."""
-    w = bi.tiny_workload(T=4, P=4, b=64, rows=500, dim=16, lengths="poisson10")
+def host_delays(P, n_iter, fixed_ns, span_ns, seed):
+    """The delays the device draws, reproduced on the host: delay of rank r before iteration j =
+    fixed + (SplitMix64 output for state seed + ((r << 40) + j + 1) * golden ratio) mod (span + 1)."""
+    r = np.arange(P, dtype=np.uint64).reshape(P, 1)
+    j = np.arange(n_iter, dtype=np.uint64).reshape(1, n_iter)
+    with np.errstate(over="ignore"):
+        z = np.uint64(seed) + ((r << np.uint64(40)) + j + np.uint64(1)) * np.uint64(0x9E3779B97F4A7C15)
+        z = (z ^ (z >> np.uint64(30))) * np.uint64(0xBF58476D1CE4E5B9)
+        z = (z ^ (z >> np.uint64(27))) * np.uint64(0x94D049BB133111EB)
+        z = z ^ (z >> np.uint64(31))
+    return fixed_ns + (z % np.uint64(span_ns + 1)).astype(np.float64)
+
+
+def timed_loop(w, tabs, d_in, k, n_iter, span_ns=0, seed=0, ring=1):
+    plan = make_plan(w, tabs, k)
+    bls.bls_set_ring(plan, ring)
+    for r in range(w.P):
+        bls.bls_set_random_stall(plan, r, span_ns, seed=seed)
+    got = []
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    e0.record()
+    for t in range(n_iter):
+        out, it = bls.bls_step(plan, k, *d_in[t])
+        if out is not None:
+            got.append(out.clone())
+    while True:
+        out, it = bls.bls_drain(plan)
+        if out is None:
+            break
+        got.append(out.clone())
+    e1.record()
+    torch.cuda.synchronize()
+    status, lag = bls.bls_status(plan)
+    return plan, got, e0.elapsed_time(e1) * 1e3 / n_iter, status, lag        # us per iteration
+
+
+@pytest.mark.parametrize("part", ["table_rr", "row_block"])
+def test_random_delays_follow_the_timing_model(part):
+    """Section V-E setting 2 / Section VI-B: every rank is delayed by a uniform random time before
+    each iteration.  Bound 0 pays the largest of the P delays in every iteration; a bound k > 0
+    lets ranks drift apart and hides the difference between the largest and the mean delay, most
+    of it already at k = 1.  The measured time per iteration is compared with the oracle's timing
+    recursion of Listing 2 fed with the very delays the device draws; every handed-back iteration
+    is compared with the oracle's pooled output."""
+    from oracle.ring_model import makespan
+    P = 8
+    w = bi.tiny_workload(T=8, P=P, b=32, rows=500, dim=16, partition=part, lengths="poisson10")
     data = [bi.table_values(t) for t in w.tables]
     tabs = dev_tables(w, data)
-    n_iter, span = 40, 400_000                                  # delays uniform in [0, 400 us]
+    n_iter, span, seed = 120, 600_000, 1234                       # delays uniform in [0, 600 us], mean D = 300 us
     inputs = [bi.make_iteration(w, t) for t in range(n_iter)]
     d_in = [(torch.from_numpy(i).cuda(), torch.from_numpy(o).cuda()) for i, o in inputs]
-    times, outs = {}, {}
-    for k in (0, 4):
+    timed_loop(w, tabs, d_in, 0, 20)                              # warm-up
+    _, _, work_us, status, _ = timed_loop(w, tabs, d_in, 0, n_iter)
+    assert status == bls.BLS_OK and work_us < 100, work_us       # stall-free time per iteration
+    delays_us = host_delays(P, n_iter, 0, span, seed) / 1e3
+    model = {k: makespan(delays_us, k, work=work_us) / n_iter for k in (0, 1, 4, 64)}
+    # closed form for bound 0: work + E[max of P uniform delays] = W + 2 D P / (P + 1)
+    assert abs(model[0] - (work_us + 600.0 * P / (P + 1))) < 0.08 * model[0]
+    times, ref = {}, None
+    for k in (0, 1, 4):
+        plan, got, us, status, lag = timed_loop(w, tabs, d_in, k, n_iter, span, seed)
+        assert status == bls.BLS_OK and lag <= k and len(got) == n_iter
+        assert_matches_oracle(w, data, inputs, got)
+        if ref is None:
+            ref = got
+        assert all(torch.equal(a, b) for a, b in zip(ref, got))  # and bit-identical for every bound
+        times[k] = us
+        assert abs(us - model[k]) <= 0.10 * model[k], (k, us, model)
+        # the stamps obey the ring's rules (checked against the same rules the oracle's RingModel enforces)
+        check_timeline(plan, w.P, k, n_iter)
+    # most of what any bound can hide is hidden by k = 1
+    assert (times[0] - times[1]) >= 0.5 * (times[0] - model[64]), (times, model)
+    assert times[4] <= times[1] * 1.02
+
+
+def check_timeline(plan, P, k, n_iter):
+    """Time stamps of post / serve / completion per (iteration, rank): an owner answers after all
+    ranks have posted, a rank completes after all owners have answered and in issue order, a rank
+    posts iteration j only after every rank has completed j - k - 1, and at no moment is the newest
+    posted iteration more than k ahead of the oldest incomplete one."""
+    post, serve, done = (a.astype(np.int64) for a in bls.bls_timeline(plan, 0, n_iter))
+    assert post.min() > 0 and serve.min() > 0 and done.min() > 0
+    assert np.all(serve >= post.max(axis=1, keepdims=True))
+    assert np.all(done >= serve.max(axis=1, keepdims=True))
+    assert np.all(np.diff(done, axis=0) >= 0) and np.all(np.diff(post, axis=0) >= 0)      # FIFO per rank
+    if n_iter > k + 1:
+        assert np.all(post[k + 1:] >= done[:n_iter - k - 1].max(axis=1, keepdims=True))   # the slot was free
+    ev = [(done[j, r], 0, r, j) for j in range(n_iter) for r in range(P)] + \
+         [(post[j, r], 1, r, j) for j in range(n_iter) for r in range(P)]
+    posted, finished, worst = [0] * P, [0] * P, 0
+    for _, kind, r, j in sorted(ev):
+        if kind == 0:
+            finished[r] = j + 1
+        else:
+            posted[r] = j + 1
+        worst = max(worst, max(posted) - 1 - min(finished))
+    assert worst <= k, worst
+
+
+def test_constant_straggler_is_not_masked_but_costs_nothing_extra():
+    """Section IV (last paragraph) / Section VI-B: one rank that is slower in every iteration sets the
+    pace whatever the bound; a bound k >= 1 must not make the loop slower than k = 0."""
+    w = bi.tiny_workload(T=4, P=4, b=64, rows=500, dim=16, partition="row_block", lengths="poisson10")
+    data = [bi.table_values(t) for t in w.tables]
+    tabs = dev_tables(w, data)
+    n_iter = 40
+    inputs = [bi.make_iteration(w, t) for t in range(n_iter)]
+    d_in = [(torch.from_numpy(i).cuda(), torch.from_numpy(o).cuda()) for i, o in inputs]
+    times = {}
+    for k in (0, 1, 4):
         plan = make_plan(w, tabs, k)
         for r in range(w.P):
-            bls.bls_set_random_stall(plan, r, span, seed=1234)
-        bls.bls_set_waves_per_step(plan, w.P + 1)               # one wave per rank that may act, plus the forcing one
+            bls.bls_set_stall(plan, r, 400_000 if r == w.P - 1 else 200_000)
         got = []
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         torch.cuda.synchronize()
@@ -251,14 +355,11 @@ def test_random_delays_are_masked_by_the_bound():
             got.append(out.clone())
         e1.record()
         torch.cuda.synchronize()
-        status, lag = bls.bls_status(plan)
-        assert status == bls.BLS_OK and lag <= k and len(got) == n_iter
+        assert bls.bls_status(plan)[0] == bls.BLS_OK
         assert_matches_oracle(w, data, inputs, got)
-        times[k], outs[k] = e0.elapsed_time(e1) / n_iter, got
-    assert all(torch.equal(a, b) for a, b in zip(outs[0], outs[4]))
-    # bound 0: about the mean of the maximum of four delays (320 us) per iteration
-    assert times[0] > 0.25
-    assert times[4] < 0.9 * times[0], times
+        times[k] = e0.elapsed_time(e1) * 1e3 / n_iter
+    assert times[0] >= 400 and times[1] >= 400 and times[4] >= 400, times     # never faster than the straggler
+    assert times[1] <= times[0] * 1.01 and times[4] <= times[0] * 1.01, times
 
 
 def test_largest_ring():
