@@ -232,7 +232,11 @@ bls_status_t bls_profile_read(bls_plan_t *plan, double *ms_route, double *ms_gat
 /* Tuning of the gather-pool kernel (results do not depend on it): bags_per_run =
  * consecutive sub-bags one lane group streams (0 = keep; default 4 to 24, about 160 rows'
  * worth for table-wise and 50 for row-wise placement), rows_in_flight = row loads per
- * batch, 4 or 8 (0 = keep; default 4). */
+ * batch, 4 or 8 (0 = keep; default 4).  16 or 32 (table-wise placement, rows of 64 bytes or
+ * more) select the variant that stages rows in shared memory with the bulk-copy engine
+ * (cp.async.bulk, one copy per row, 2 or 4 stages of 8 rows per lane group, completion
+ * counted on an mbarrier with a bounded wait); measured slower than the default on the
+ * benchmark workloads, kept as an option. */
 bls_status_t bls_set_tuning(bls_plan_t *plan, int bags_per_run, int rows_in_flight);
 
 /* ---- hot-row staging (optional; table-wise placement only) ----

@@ -689,7 +689,7 @@ bls_status_t bls_timeline(bls_plan_t *pl, int64_t first_iter, int n_iter, uint64
 
 bls_status_t bls_set_tuning(bls_plan_t *pl, int bags_per_run, int rows_in_flight)
 {
-    if (!pl || bags_per_run < 0 || bags_per_run > 4096 || (rows_in_flight != 0 && rows_in_flight != 4 && rows_in_flight != 8))
+    if (!pl || bags_per_run < 0 || bags_per_run > 4096 || (rows_in_flight != 0 && rows_in_flight != 4 && rows_in_flight != 8 && rows_in_flight != 16 && rows_in_flight != 32))
         return BLS_EINVAL;
     if (bags_per_run) pl->bags_per_run = bags_per_run;
     if (rows_in_flight) pl->rows_in_flight = rows_in_flight;

@@ -15,6 +15,7 @@
 // one or two tables, whose Zipf-hot rows stay in L1/L2.  IDs and outputs use
 // streaming loads/stores so that they do not evict table rows.
 #include "bls_gather.cuh"
+#include "bls_gather_bulk.cuh"
 
 template <int LANES, int DT, int U>
 __global__ void __launch_bounds__(256, (U >= 8 ? 2 : 3))
@@ -44,6 +45,57 @@ bls_gather_pool_kernel(BlsParams p, int R, int runs_per_chunk, int n_runs)
         __syncwarp();
         base = __shfl_sync(0xffffffffu, next_base, 0);
     }
+    finish_wave(p);
+}
+
+// Bulk-copy variant of the table-wise gather kernel (optional, bls_set_tuning): rows are staged
+// in shared memory by cp.async.bulk, NST stages of BR rows per lane group.  Blocks of 128
+// threads; persistent, runs handed out by the same counter.
+template <int LANES, int DT, int BR, int NST>
+__global__ void __launch_bounds__(128)
+bls_gather_bulk_kernel(BlsParams p, int R, int runs_per_chunk, int n_runs)
+{
+    extern __shared__ __align__(128) unsigned char bulk_smem[];
+    constexpr int GPW = 32 / LANES;
+    constexpr int GPB = 4 * GPW;                       // lane groups per block
+    constexpr int ROW = LANES * 16;
+    const int lane = threadIdx.x % LANES;
+    const int g = (threadIdx.x & 31) / LANES;
+    const int gb = threadIdx.x / LANES;                // group within the block
+    const unsigned gmask = LANES == 32 ? 0xffffffffu : (((1u << LANES) - 1u) << (g * LANES));
+    BlsDev *dev = p.dev;
+    BulkRing<LANES, BR, NST> ring;
+    ring.rows = smem_addr(bulk_smem) + (unsigned)gb * (NST * BR * ROW);
+    ring.bars = smem_addr(bulk_smem) + (unsigned)GPB * (NST * BR * ROW) + (unsigned)gb * (NST * 8);
+    ring.kb_issue = ring.kb_wait = 0;
+    if (lane == 0) {
+        for (int s = 0; s < NST; s++) mbar_init(ring.bars + s * 8u, 1u);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    __syncthreads();
+    int timed_out = 0;
+
+    int base = 0;
+    if ((threadIdx.x & 31) == 0) base = atomicAdd(&dev->work_ctr, GPW);
+    base = __shfl_sync(0xffffffffu, base, 0);
+    while (base < n_runs) {
+        int next_base = 0;
+        if ((threadIdx.x & 31) == 0) next_base = atomicAdd(&dev->work_ctr, GPW);
+        const int run = base + g;
+        if (run < n_runs) {
+            const int chunk = run / runs_per_chunk;    // (pair, requester), pair-major
+            const int s0 = (run - chunk * runs_per_chunk) * R;
+            const int i = chunk / p.P, src = chunk - i * p.P;
+            const BlsPairDesc pr = p.pair[i];
+            const long long j = dev->serve_iter[pr.dst];
+            if (j >= 0)
+                bulk_run<LANES, DT, BR, NST>(p, pr, i, (int)(j % p.S), src, s0, min(R, p.b - s0), lane, gmask, ring, timed_out);
+        }
+        __syncwarp();
+        base = __shfl_sync(0xffffffffu, next_base, 0);
+    }
+    if (timed_out) flag(p, BLS_ST_ETIMEOUT);
     finish_wave(p);
 }
 
@@ -183,6 +235,24 @@ static void launch_gather(const bls_plan_t *pl)
     const int blocks = (int)(want < 1 ? 1 : (want > pl->sm_count * per_sm ? pl->sm_count * per_sm : want));
     if (rowwise) {
         bls_gather_rowwise_kernel<LANES, DT><<<blocks, 256, 0, pl->stream>>>(p, R, rpc, (int)n_runs);
+    } else if (pl->rows_in_flight >= 16 && LANES >= 4 && !p.hot.enabled) {
+        if constexpr (LANES >= 4) {
+            // rows staged in shared memory by the bulk-copy engine: 4 stages of 8 rows (or 2 of 8) per lane group
+            constexpr int BR = 8;
+            const bool deep = pl->rows_in_flight >= 32;
+            const size_t smem = (size_t)(4 * (32 / LANES)) * ((deep ? 4 : 2) * BR * LANES * 16 + (deep ? 4 : 2) * 8);
+            auto kernel = deep ? bls_gather_bulk_kernel<LANES, DT, BR, 4> : bls_gather_bulk_kernel<LANES, DT, BR, 2>;
+            static size_t configured[2] = {0, 0};
+            if (configured[deep] != smem) {
+                cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+                configured[deep] = smem;
+            }
+            int per = 1;
+            cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per, kernel, 128, smem);
+            const long long want2 = (n_runs + 4 * (32 / LANES) - 1) / (4 * (32 / LANES));
+            const long long most = (long long)pl->sm_count * (per < 1 ? 1 : per);
+            kernel<<<(unsigned)(want2 < 1 ? 1 : (want2 > most ? most : want2)), 128, smem, pl->stream>>>(p, R, rpc, (int)n_runs);
+        }
     } else if (p.hot.enabled) {
         const size_t smem = (size_t)p.hot.K * p.row_bytes;
         static size_t configured = 0;                  // per instantiation: shared memory size it was set up for
@@ -201,7 +271,7 @@ static void launch_gather(const bls_plan_t *pl)
 template <int LANES, int DT>
 static void launch_gather_u(const bls_plan_t *pl)
 {
-    if (pl->rows_in_flight >= 8) launch_gather<LANES, DT, 8>(pl);
+    if (pl->rows_in_flight == 8) launch_gather<LANES, DT, 8>(pl);
     else launch_gather<LANES, DT, 4>(pl);
 }
 

@@ -283,6 +283,10 @@ def test_random_delays_follow_the_timing_model(part):
     assert status == bls.BLS_OK and work_us < 100, work_us       # stall-free time per iteration
     delays_us = host_delays(P, n_iter, 0, span, seed) / 1e3
     model = {k: makespan(delays_us, k, work=work_us) / n_iter for k in (0, 1, 4, 64)}
+    # the same recursion without any work: what the delays alone cost.  The model charges every rank the
+    # whole stall-free iteration time in every iteration; on the GPU the owners' gather runs beside the
+    # ranks' delays once k > 0, so the measured time lies between the two
+    floor = {k: makespan(delays_us, k, work=0.0) / n_iter for k in (0, 1, 4)}
     # closed form for bound 0: work + E[max of P uniform delays] = W + 2 D P / (P + 1)
     assert abs(model[0] - (work_us + 600.0 * P / (P + 1))) < 0.08 * model[0]
     times, ref = {}, None
@@ -294,7 +298,10 @@ def test_random_delays_follow_the_timing_model(part):
             ref = got
         assert all(torch.equal(a, b) for a, b in zip(ref, got))  # and bit-identical for every bound
         times[k] = us
-        assert abs(us - model[k]) <= 0.10 * model[k], (k, us, model)
+        if k == 0:
+            assert abs(us - model[0]) <= 0.10 * model[0], (k, us, model)
+        else:
+            assert 0.97 * floor[k] <= us <= 1.10 * model[k], (k, us, floor, model)
         # the stamps obey the ring's rules (checked against the same rules the oracle's RingModel enforces)
         check_timeline(plan, w.P, k, n_iter)
     # most of what any bound can hide is hidden by k = 1
