@@ -307,6 +307,41 @@ bls_status_t bls_a2a_wait(bls_a2a_t *handle, const void **recv /*host out*/, int
                           int64_t *request /*host out*/);
 bls_status_t bls_a2a_status(bls_a2a_t *handle);
 
+/* ---- the dense stages either side of the lookup (Section IV, Listing 1 / Listing 2) ----
+ * Listing 1 runs the bottom MLP on the dense features between the alltoall and its wait, then
+ * the feature interaction of its output with the pooled vectors and the top MLP; Listing 2 lets
+ * those stages of batch j run beside the exchange of later batches (Table I).  These calls are
+ * stand-ins for those stages with weights the caller provides (the paper takes them from the
+ * reference DLRM and does not restate them); all buffers are DEVICE memory.
+ *
+ * An MLP is n_layers linear layers y = act(x W^T + bias): dims[0] inputs, dims[i+1] outputs of
+ * layer i; weights[i] is bf16 [dims[i+1]][dims[i]] row-major, 16-byte aligned; bias[i] fp32
+ * [dims[i+1]]; every dims[i] with i < n_layers is a multiple of 8.  Hidden layers use ReLU, the
+ * last layer last_act (0 none, 1 ReLU, 2 logistic function).  Activations are bf16 between
+ * layers, sums are fp32 (tensor cores: tcgen05.mma fed by TMA tile loads, accumulator in tensor
+ * memory).  The workspace (bls_mlp_bytes, 256-byte aligned, borrowed until bls_mlp_destroy)
+ * holds the hidden activations of up to max_rows rows; weights and biases are borrowed too.
+ *   bls_mlp_forward  x bf16 [rows][ldx] (ldx a multiple of 8, >= dims[0], 16-byte aligned base)
+ *                    -> y [rows][ldy]: bf16, or fp32 when y_fp32.  Asynchronous on cuda_stream;
+ *                    calls that use the same handle must not overlap on the GPU.
+ *   bls_interact     x bf16 [rows][ldx] (the bottom MLP's output, D columns used), pooled fp32
+ *                    [rows][T][D] (a slot of the ring: out[src][s][t][:] is [rows = P*b][T][D])
+ *                    -> r bf16 [rows][ldr]: the D values of x, then the dot products
+ *                    <v_i, v_j>, i = 1..T, j < i, of v_0 = x and v_1..v_T = the pooled vectors
+ *                    (strictly lower triangle, row-major), then zeros up to ldr
+ *   bls_mlp_status   synchronises cuda_stream; BLS_ETIMEOUT if a bounded wait inside a kernel gave up */
+typedef struct bls_mlp bls_mlp_t;
+bls_status_t bls_mlp_bytes(int n_layers, const int *dims /*host*/, int max_rows, size_t *bytes /*host*/);
+bls_status_t bls_mlp_create(int n_layers, const int *dims /*host*/, const void *const *weights /*host array of device ptrs*/,
+                            const float *const *bias /*host array of device ptrs*/, int last_act, int max_rows,
+                            void *workspace, size_t bytes, void *cuda_stream, bls_mlp_t **handle /*host out*/);
+void bls_mlp_destroy(bls_mlp_t *handle);
+bls_status_t bls_mlp_forward(bls_mlp_t *handle, const void *x, int ldx, int rows, void *y, int ldy, int y_fp32,
+                             void *cuda_stream);
+bls_status_t bls_interact(const void *x, int ldx, const float *pooled, int rows, int T, int D, void *r, int ldr,
+                          void *cuda_stream);
+bls_status_t bls_mlp_status(bls_mlp_t *handle, void *cuda_stream);
+
 /* ---- allocation-free router (the paper has no counterpart: this entry point
  * exists for deployment reasons only) ----
  * Step (1) for table-wise round-robin placement, for callers that cannot

@@ -26,7 +26,8 @@ EXPORTS = ["bls_plan_bytes", "bls_plan", "bls_destroy", "bls_route", "bls_lookup
            "bls_set_stall", "bls_set_wait_limit", "bls_strerror", "bls_fill_hash_table",
            "bls_profile", "bls_profile_read", "bls_set_tuning", "bls_route_table_rr_static",
            "bls_set_random_stall", "bls_set_ring", "bls_timeline", "bls_set_poison", "bls_set_overlap", "bls_a2a_bytes", "bls_a2a_create", "bls_a2a_destroy", "bls_a2a_post", "bls_a2a_wait",
-           "bls_a2a_status", "bls_hot_bytes", "bls_hot_attach", "bls_hot_observe", "bls_hot_build", "bls_hot_view"]
+           "bls_a2a_status", "bls_mlp_bytes", "bls_mlp_create", "bls_mlp_destroy", "bls_mlp_forward", "bls_interact",
+           "bls_mlp_status", "bls_hot_bytes", "bls_hot_attach", "bls_hot_observe", "bls_hot_build", "bls_hot_view"]
 
 
 class BlsError(RuntimeError):
@@ -366,3 +367,55 @@ class A2a:
                 lib().bls_a2a_destroy(h)
             except Exception:
                 pass
+
+
+class Mlp:
+    """Handle of a stand-in MLP stage (bottom or top MLP of Listing 1 / Listing 2).
+
+    weights[i]: bf16 [dims[i+1]][dims[i]] device tensors, biases[i]: fp32 [dims[i+1]]; hidden layers
+    use ReLU, the last one last_act (0 none, 1 ReLU, 2 logistic function)."""
+
+    def __init__(self, weights: Sequence[torch.Tensor], biases: Sequence[torch.Tensor], last_act: int, max_rows: int,
+                 stream: Optional[torch.cuda.Stream] = None):
+        n = len(weights)
+        self.dims = [weights[0].shape[1]] + [w.shape[0] for w in weights]
+        for w, b in zip(weights, biases):
+            if w.dtype != torch.bfloat16 or b.dtype != torch.float32 or not w.is_contiguous() or not b.is_contiguous():
+                raise ValueError("weights must be contiguous bf16 [out][in], biases contiguous fp32")
+        dims = (C.c_int * (n + 1))(*self.dims)
+        nbytes = C.c_size_t(0)
+        _check(lib().bls_mlp_bytes(n, dims, max_rows, C.byref(nbytes)), "bls_mlp_bytes")
+        ws = torch.empty(nbytes.value + 256, dtype=torch.uint8, device=weights[0].device)
+        pad = (-ws.data_ptr()) % 256
+        self.workspace = ws[pad:pad + nbytes.value]
+        self.weights, self.biases, self.max_rows = list(weights), list(biases), max_rows
+        wp = (C.c_void_p * n)(*[w.data_ptr() for w in weights])
+        bp = (C.c_void_p * n)(*[b.data_ptr() for b in biases])
+        self.handle = C.c_void_p()
+        _check(lib().bls_mlp_create(n, dims, wp, bp, last_act, max_rows, C.c_void_p(self.workspace.data_ptr()),
+                                    C.c_size_t(nbytes.value), _stream_ptr(stream), C.byref(self.handle)), "bls_mlp_create")
+
+    def forward(self, x: torch.Tensor, y: torch.Tensor, stream: Optional[torch.cuda.Stream] = None) -> None:
+        """x bf16 [rows][ldx] -> y [rows][ldy] (bf16 or fp32); asynchronous on the stream."""
+        _check(lib().bls_mlp_forward(self.handle, C.c_void_p(x.data_ptr()), x.stride(0), x.shape[0],
+                                     C.c_void_p(y.data_ptr()), y.stride(0), int(y.dtype == torch.float32),
+                                     _stream_ptr(stream)), "bls_mlp_forward")
+
+    def status(self, stream: Optional[torch.cuda.Stream] = None) -> int:
+        return lib().bls_mlp_status(self.handle, _stream_ptr(stream))
+
+    def __del__(self):
+        h, self.handle = getattr(self, "handle", None), None
+        if h:
+            try:
+                lib().bls_mlp_destroy(h)
+            except Exception:
+                pass
+
+
+def bls_interact(x: torch.Tensor, pooled: torch.Tensor, r: torch.Tensor, stream: Optional[torch.cuda.Stream] = None) -> None:
+    """x bf16 [rows][>=D], pooled fp32 [rows][T][D] (or any shape with rows*T*D elements in that order), r bf16 [rows][ldr]."""
+    rows, D = x.shape[0], pooled.shape[-1]
+    T = pooled.numel() // (rows * D)
+    _check(lib().bls_interact(C.c_void_p(x.data_ptr()), x.stride(0), C.c_void_p(pooled.data_ptr()), rows, T, D,
+                              C.c_void_p(r.data_ptr()), r.stride(0), _stream_ptr(stream)), "bls_interact")
