@@ -61,6 +61,9 @@ def parse_args():
     ap.add_argument("--repeats", type=int, default=5,
                     help="repetitions of the timed loop at the headline bound for the mean and 95 %% confidence interval")
     ap.add_argument("--ks", default="", help="comma-separated bounds to time instead of the workload's own")
+    ap.add_argument("--stages", action="store_true",
+                    help="time the loop with the dense stages of Listing 1/2 around the lookup (bottom MLP, interaction, "
+                         "top MLP; random weights): serial, Listing 1's overlap at k = 0, and Listing 2's at k >= 1")
     ap.add_argument("--ring", type=int, default=None, choices=[-1, 0, 1],
                     help="persistent ring kernel: -1 only with injected delays, 0 also for small iterations, 1 always "
                          "(default: the library's own choice)")
@@ -638,10 +641,154 @@ def run_a2a(args):
                       "note": "GB/s counts bytes read plus bytes written; one post kernel and one completion kernel per call"}))
 
 
+def run_stages(args):
+    """Listing 1 / Listing 2 with real compute around the lookup (Table I's overlap classes).
+
+    serial      bottom MLP, lookup, interaction and top MLP one after the other on one stream (k = 0)
+    listing1    k = 0, the bottom MLP of batch t on a second stream beside the lookup of batch t
+                (computation and communication of the same batch overlap)
+    listing2    k >= 1: in addition the interaction and top MLP of batch t - k run on a third stream
+                beside the lookup of batch t + 1 (computation of one batch beside communication of another)
+    """
+    import torch
+    import paper_2512_19342_b200 as bls
+    torch.cuda.set_device(0)
+    w = select(bi.workload(args.config), args)
+    nd = N_DISTINCT[args.config]
+    inputs = host_inputs(w, nd)
+    tabs = device_tables(w, bls, torch)
+    d_in = [(torch.from_numpy(i).cuda(), torch.from_numpy(o).cuda()) for i, o in inputs]
+    P, T, b, D = w.P, w.T, w.local_batch, w.tables[0].dim
+    B = P * b
+    k_max = max(max(w.ks), 1)
+    plan = bls.bls_plan(tabs, w.partition, P, b, k_max, capacity(w, inputs))
+    g = torch.Generator(device="cuda").manual_seed(1)
+
+    def mlp(dims, last_act):
+        ws = [(torch.randn(dims[i + 1], dims[i], device="cuda", generator=g) / dims[i] ** 0.5).to(torch.bfloat16)
+              for i in range(len(dims) - 1)]
+        bs = [torch.zeros(dims[i + 1], device="cuda") for i in range(len(dims) - 1)]
+        return bls.Mlp(ws, bs, last_act, B)
+
+    n_int = D + T * (T + 1) // 2
+    ldr = (n_int + 63) // 64 * 64
+    bot = mlp([16, 512, 256, D], 1)
+    top = mlp([ldr, 512, 256, 8], 2)
+    flops = 2.0 * B * (16 * 512 + 512 * 256 + 256 * D + ldr * 512 + 512 * 256 + 256 * 8)
+    dense = torch.randn(B, 16, device="cuda", generator=g).to(torch.bfloat16)
+    S = k_max + 1
+    xs = [torch.empty(B, D, dtype=torch.bfloat16, device="cuda") for _ in range(S)]
+    rs = [torch.empty(B, ldr, dtype=torch.bfloat16, device="cuda") for _ in range(2)]
+    ps = [torch.empty(B, 8, dtype=torch.float32, device="cuda") for _ in range(2)]
+    main = torch.cuda.current_stream()
+    s_bot, s_top = torch.cuda.Stream(), torch.cuda.Stream()
+
+    def loop(mode, k, steps):
+        ev_bot = [None] * S
+        ev_top = [None, None]
+        n_top = 0
+
+        def tail(out, it, stream):
+            nonlocal n_top
+            q = n_top & 1
+            n_top += 1
+            if ev_bot[it % S] is not None:
+                stream.wait_event(ev_bot[it % S])
+            bls.bls_interact(xs[it % S], out, rs[q], stream)
+            top.forward(rs[q], ps[q], stream)
+            if stream is not main:
+                ev_top[q] = torch.cuda.Event()
+                ev_top[q].record(stream)
+
+        for t in range(steps):
+            ids, off = d_in[t % nd]
+            if mode == "serial":
+                bot.forward(dense, xs[t % S], main)
+            else:
+                e = torch.cuda.Event()
+                e.record(main)
+                s_bot.wait_event(e)
+                bot.forward(dense, xs[t % S], s_bot)
+                ev_bot[t % S] = torch.cuda.Event()
+                ev_bot[t % S].record(s_bot)
+            for e in ev_top:                       # the slot the next answer goes to, and r / p, are free again
+                if e is not None:
+                    main.wait_event(e)
+            out, it = bls.bls_step(plan, k, ids, off)
+            if out is not None:
+                if mode == "listing2":
+                    e = torch.cuda.Event()
+                    e.record(main)
+                    s_top.wait_event(e)
+                    tail(out, it, s_top)
+                else:
+                    tail(out, it, main)
+        while True:
+            out, it = bls.bls_drain(plan)
+            if out is None:
+                break
+            tail(out, it, main)
+        for e in ev_top:
+            if e is not None:
+                main.wait_event(e)
+        main.wait_stream(s_bot)
+
+    def timed(mode, k, steps):
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        loop(mode, k, steps)
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / steps
+
+    def timed_plain(k, steps):                     # the lookup alone
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for t in range(steps):
+            bls.bls_step(plan, k, *d_in[t % nd])
+        while bls.bls_drain(plan)[0] is not None:
+            pass
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / steps
+
+    def timed_dense(steps):                        # the dense stages alone, on one stream
+        pooled = torch.randn(B, T, D, device="cuda", generator=g)
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for t in range(steps):
+            bot.forward(dense, xs[0], main)
+            bls.bls_interact(xs[0], pooled, rs[0], main)
+            top.forward(rs[0], ps[0], main)
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / steps
+
+    n = args.steps
+    loop("serial", 0, 5)
+    res = {"mode": "stages", "workload": w.name, "steps": n, "rows": B, "dense_flops_per_step": flops,
+           "lookup_only_ms": {"0": timed_plain(0, n), str(k_max): timed_plain(k_max, n)},
+           "dense_only_ms": timed_dense(n)}
+    res["dense_only_tflops"] = flops / (res["dense_only_ms"] * 1e-3) / 1e12
+    res["serial_k0_ms"] = timed("serial", 0, n)
+    res["listing1_k0_ms"] = timed("listing1", 0, n)
+    for k in sorted({1, k_max}):
+        res[f"listing2_k{k}_ms"] = timed("listing2", k, n)
+    assert bls.bls_status(plan)[0] == bls.BLS_OK and bot.status() == bls.BLS_OK and top.status() == bls.BLS_OK
+    res["probability_sample"] = [float(x) for x in ps[0][:4, 0].cpu()]
+    print(json.dumps(res))
+
+
 def main():
     args = parse_args()
     if args.a2a:
         run_a2a(args)
+        return
+    if args.stages:
+        run_stages(args)
         return
     if args.impl == "reference":
         run_reference(args)

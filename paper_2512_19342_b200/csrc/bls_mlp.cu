@@ -26,7 +26,7 @@ namespace {
 
 constexpr int MLP_BM = 128;          // rows of Y per CTA (= TMEM lanes)
 constexpr int MLP_BK = 64;           // K per stage: 64 bf16 = 128 bytes = one swizzle span
-constexpr int MLP_STAGES = 4;
+constexpr int MLP_STAGES = 3;          // 3 x 32 KiB of tiles at BN = 128: two CTAs per SM, one computes while the other stores
 constexpr int MLP_THREADS = 192;     // warp 0: TMA, warp 1: MMA + TMEM allocation, warps 2-5: epilogue
 
 __device__ __forceinline__ unsigned long long mlp_clock()
@@ -186,24 +186,35 @@ bls_linear_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
         const int row = m0 + q * 32 + lane;
         if (mb_wait(done_bar, 0, a.status)) {
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+            // bf16 output with whole 16-byte pieces: the warp's 32 x BN block goes through shared memory (the
+            // tile ring is free: every MMA that read it has completed) and leaves as coalesced row pieces
+            const bool staged = !a.y_fp32 && (a.ldy & 7) == 0 && (a.N & 7) == 0;
+            constexpr int ROWB = BN * 2;                                      // bytes of one staged row
+            const unsigned stage = tiles + (unsigned)q * 32u * ROWB;
             #pragma unroll 1
             for (int c0 = 0; c0 < BN; c0 += 32) {
                 unsigned r[32];
                 tmem_ld32(tmem + ((unsigned)(q * 32) << 16) + (unsigned)c0, r);   // sync.aligned: the whole warp, also rows past M
-                if (row < a.M && !a.y_fp32 && n0 + c0 + 32 <= a.N && (a.ldy & 7) == 0) {
-                    // a whole chunk of bf16 output: 64 contiguous bytes of the row, four 16-byte stores
-                    unsigned pk[16];
+                if (staged) {
                     #pragma unroll
-                    for (int j = 0; j < 32; j += 2) {
-                        float v0 = __uint_as_float(r[j]) + a.bias[n0 + c0 + j], v1 = __uint_as_float(r[j + 1]) + a.bias[n0 + c0 + j + 1];
-                        if (a.act == 1) { v0 = fmaxf(v0, 0.f); v1 = fmaxf(v1, 0.f); }
-                        else if (a.act == 2) { v0 = 1.f / (1.f + expf(-v0)); v1 = 1.f / (1.f + expf(-v1)); }
-                        __nv_bfloat162 h2 = __floats2bfloat162_rn(v0, v1);
-                        pk[j >> 1] = *reinterpret_cast<unsigned *>(&h2);
+                    for (int j = 0; j < 32; j += 8) {
+                        unsigned pk[4];
+                        #pragma unroll
+                        for (int e = 0; e < 8; e += 2) {
+                            const int col = n0 + c0 + j + e;
+                            float v0 = __uint_as_float(r[j + e]) + (col < a.N ? a.bias[col] : 0.f);
+                            float v1 = __uint_as_float(r[j + e + 1]) + (col + 1 < a.N ? a.bias[col + 1] : 0.f);
+                            if (a.act == 1) { v0 = fmaxf(v0, 0.f); v1 = fmaxf(v1, 0.f); }
+                            else if (a.act == 2) { v0 = 1.f / (1.f + expf(-v0)); v1 = 1.f / (1.f + expf(-v1)); }
+                            __nv_bfloat162 h2 = __floats2bfloat162_rn(v0, v1);
+                            pk[e >> 1] = *reinterpret_cast<unsigned *>(&h2);
+                        }
+                        // 16-byte piece number (c0 + j) / 8 of the row, rotated by the row number so that the
+                        // lanes of a warp (32 different rows, same piece) hit different banks
+                        const unsigned piece = ((unsigned)((c0 + j) >> 3) + (unsigned)lane) % (unsigned)(BN / 8);
+                        asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};"
+                                     ::"r"(stage + (unsigned)lane * ROWB + piece * 16u), "r"(pk[0]), "r"(pk[1]), "r"(pk[2]), "r"(pk[3]) : "memory");
                     }
-                    uint4 *dst = reinterpret_cast<uint4 *>((__nv_bfloat16 *)a.Y + (size_t)row * a.ldy + n0 + c0);
-                    #pragma unroll
-                    for (int j = 0; j < 4; j++) dst[j] = make_uint4(pk[4 * j], pk[4 * j + 1], pk[4 * j + 2], pk[4 * j + 3]);
                 } else if (row < a.M) {
                     #pragma unroll
                     for (int j = 0; j < 32; j++) {
@@ -218,6 +229,21 @@ bls_linear_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
                     }
                 }
             }
+            if (staged) {
+                __syncwarp();
+                constexpr int PPR = BN / 8;                                   // 16-byte pieces per row
+                for (int e = lane; e < 32 * PPR; e += 32) {
+                    const int rr = e / PPR, pc = e % PPR;                     // row of the block, piece of the row
+                    const int grow = m0 + q * 32 + rr, col = n0 + pc * 8;
+                    if (grow < a.M && col < a.N) {                            // N and ldy are multiples of 8: a piece is inside or outside
+                        const unsigned piece = ((unsigned)pc + (unsigned)rr) % (unsigned)PPR;
+                        uint4 v;
+                        asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];"
+                                     : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(stage + (unsigned)rr * ROWB + piece * 16u));
+                        *reinterpret_cast<uint4 *>((__nv_bfloat16 *)a.Y + (size_t)grow * a.ldy + col) = v;
+                    }
+                }
+            }
         }
     }
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
@@ -228,31 +254,70 @@ bls_linear_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
     }
 }
 
-// Feature interaction, one block per sample: v_0 = the bottom MLP's output (bf16), v_1..v_T =
-// the pooled vectors (fp32); R = [v_0, <v_i, v_j> for i = 1..T, j < i], bf16, zero-padded to ldr.
-__global__ void __launch_bounds__(128) bls_interact_kernel(const __nv_bfloat16 *x, int ldx, const float *pooled, int B, int T, int D,
-                                                           __nv_bfloat16 *r, int ldr)
+// Feature interaction, one block of 64 threads per sample: v_0 = the bottom MLP's output (bf16),
+// v_1..v_T = the pooled vectors (fp32); R = [v_0, <v_i, v_j> for i = 1..T, j < i], bf16, zero-padded
+// to ldr.  The vectors are staged in shared memory; a thread computes a 3 x 3 block of the matrix of
+// dot products (only blocks on or below the diagonal exist), so every value read from shared
+// memory is used three times.
+__global__ void __launch_bounds__(64) bls_interact_kernel(const __nv_bfloat16 *x, int ldx, const float *pooled, int B, int T, int D,
+                                                          __nv_bfloat16 *r, int ldr)
 {
-    extern __shared__ float iv[];                      // [T + 1][D + 1] (padded rows: no bank conflicts between vectors)
+    extern __shared__ float iv[];                      // [3 * nb][D + 1]: rows padded so that vectors start in different banks
     const int b = blockIdx.x;
     const int W = D + 1;
-    for (int e = threadIdx.x; e < (T + 1) * D; e += blockDim.x) {
-        const int i = e / D, c = e - i * D;
-        iv[i * W + c] = i == 0 ? __bfloat162float(x[(size_t)b * ldx + c]) : pooled[((size_t)b * T + (i - 1)) * D + c];
+    const int nb = (T + 1 + 2) / 3;                    // blocks of three vectors
+    for (int c = threadIdx.x; c < D; c += blockDim.x) iv[c] = __bfloat162float(x[(size_t)b * ldx + c]);
+    for (int e = (T + 1) * D + threadIdx.x; e < 3 * nb * D; e += blockDim.x) iv[(e / D) * W + e % D] = 0.f;   // rows that pad the last block
+    if ((D & 3) == 0) {
+        // the sample's T pooled vectors are one contiguous piece of T * D floats: 16-byte loads, four in flight per thread
+        const float4 *src = reinterpret_cast<const float4 *>(pooled + (size_t)b * T * D);
+        const int n4 = T * D / 4;
+        for (int e0 = threadIdx.x; e0 < n4; e0 += 4 * blockDim.x) {
+            float4 v[4];
+            #pragma unroll
+            for (int u = 0; u < 4; u++) {
+                const int e = e0 + u * blockDim.x;
+                if (e < n4) v[u] = __ldcs(src + e);
+            }
+            #pragma unroll
+            for (int u = 0; u < 4; u++) {
+                const int e = e0 + u * blockDim.x;
+                if (e < n4) {
+                    const int i = 1 + (e * 4) / D, c = (e * 4) % D;
+                    float *dst = iv + i * W + c;
+                    dst[0] = v[u].x; dst[1] = v[u].y; dst[2] = v[u].z; dst[3] = v[u].w;
+                }
+            }
+        }
+    } else {
+        for (int e = threadIdx.x; e < T * D; e += blockDim.x) iv[(1 + e / D) * W + e % D] = pooled[(size_t)b * T * D + e];
     }
     __syncthreads();
     __nv_bfloat16 *out = r + (size_t)b * ldr;
     for (int c = threadIdx.x; c < D; c += blockDim.x) out[c] = x[(size_t)b * ldx + c];
     const int npairs = T * (T + 1) / 2;
-    for (int q = threadIdx.x; q < npairs; q += blockDim.x) {
-        // pair number q -> (i, j), i = 1..T, j < i, row-major over the strictly lower triangle
-        int i = (int)((1.f + sqrtf(1.f + 8.f * (float)q)) * 0.5f);
-        while (i * (i - 1) / 2 > q) i--;
-        while ((i + 1) * i / 2 <= q) i++;
-        const int j = q - i * (i - 1) / 2;
-        float s = 0.f;
-        for (int c = 0; c < D; c++) s = fmaf(iv[i * W + c], iv[j * W + c], s);
-        out[D + q] = __float2bfloat16_rn(s);
+    for (int q = threadIdx.x; q < nb * (nb + 1) / 2; q += blockDim.x) {
+        // block pair number q -> (bi, bj), bj <= bi, row-major over the lower triangle including the diagonal
+        int bi = (int)((sqrtf(1.f + 8.f * (float)q) - 1.f) * 0.5f);
+        while (bi * (bi + 1) / 2 > q) bi--;
+        while ((bi + 1) * (bi + 2) / 2 <= q) bi++;
+        const int bj = q - bi * (bi + 1) / 2;
+        const float *pa = iv + 3 * bi * W, *pb = iv + 3 * bj * W;
+        float acc[3][3] = {};
+        for (int c = 0; c < D; c++) {
+            const float a0 = pa[c], a1 = pa[W + c], a2 = pa[2 * W + c];
+            const float b0 = pb[c], b1 = pb[W + c], b2 = pb[2 * W + c];
+            acc[0][0] = fmaf(a0, b0, acc[0][0]); acc[0][1] = fmaf(a0, b1, acc[0][1]); acc[0][2] = fmaf(a0, b2, acc[0][2]);
+            acc[1][0] = fmaf(a1, b0, acc[1][0]); acc[1][1] = fmaf(a1, b1, acc[1][1]); acc[1][2] = fmaf(a1, b2, acc[1][2]);
+            acc[2][0] = fmaf(a2, b0, acc[2][0]); acc[2][1] = fmaf(a2, b1, acc[2][1]); acc[2][2] = fmaf(a2, b2, acc[2][2]);
+        }
+        #pragma unroll
+        for (int u = 0; u < 3; u++)
+            #pragma unroll
+            for (int v = 0; v < 3; v++) {
+                const int i = 3 * bi + u, j = 3 * bj + v;
+                if (i <= T && j < i) out[D + i * (i - 1) / 2 + j] = __float2bfloat16_rn(acc[u][v]);
+            }
     }
     for (int c = D + npairs + threadIdx.x; c < ldr; c += blockDim.x) out[c] = __float2bfloat16_rn(0.f);
 }
@@ -399,9 +464,9 @@ bls_status_t bls_interact(const void *x, int ldx, const float *pooled, int rows,
                           void *cuda_stream)
 {
     if (!x || !pooled || !r || rows < 1 || T < 1 || D < 1 || ldx < D || ldr < D + T * (T + 1) / 2) return BLS_EINVAL;
-    const size_t smem = sizeof(float) * (size_t)(T + 1) * (D + 1);
+    const size_t smem = sizeof(float) * (size_t)(3 * ((T + 3) / 3)) * (D + 1);
     if (smem > 48 * 1024) return BLS_ENOSPC;
-    bls_interact_kernel<<<rows, 128, smem, (cudaStream_t)cuda_stream>>>((const __nv_bfloat16 *)x, ldx, pooled, rows, T, D,
+    bls_interact_kernel<<<rows, 64, smem, (cudaStream_t)cuda_stream>>>((const __nv_bfloat16 *)x, ldx, pooled, rows, T, D,
                                                                          (__nv_bfloat16 *)r, ldr);
     return cudaGetLastError() == cudaSuccess ? BLS_OK : BLS_ECUDA;
 }
