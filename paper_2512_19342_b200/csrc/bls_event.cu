@@ -25,6 +25,8 @@
 
 namespace {
 
+constexpr int RING_GATHER_CHUNK = 8;    // warp-sized pieces of work per gather tile (a block has 4 warps)
+
 struct RingArgs {
     int mode;                   // BLS_MODE_STEP or BLS_MODE_DRAIN
     int k;
@@ -79,23 +81,30 @@ template <int LANES, int DT, int PART>
 __device__ __forceinline__ void ring_worker(const BlsParams &p, const RingArgs &a)
 {
     constexpr int GPW = 32 / LANES;                    // runs per warp
-    constexpr int RPT = (BLS_ROUTE_TB / 32) * GPW;     // runs per gather tile
-    __shared__ int s_q, s_tile;
+    constexpr int RPT = RING_GATHER_CHUNK * GPW;       // runs per gather tile
+    __shared__ int s_q, s_tile, s_ctr;
     BlsQueue *q = p.queue;
     unsigned cur = 0;                                  // oldest action that may still have tiles (thread 0 only)
+    unsigned acquired = 0;                             // actions below this index were published before this block's last acquire
     // a worker gives up long after the scheduler would have (its limit covers the scheduler's two stages)
     const unsigned long long limit = 4ull * p.dev->wait_limit_ns + 1000000000ull;
     const int lane = threadIdx.x % LANES;
     const int g = (threadIdx.x & 31) / LANES;
-    const int warp = threadIdx.x >> 5;
     for (;;) {
         if (threadIdx.x == 0) {
             int got = -1, tile = 0;
             const unsigned long long t0 = globaltimer_ns();
             unsigned spins = 0;
             for (;;) {
-                const unsigned tail = ld_acquire(&q->tail);
+                // The tail is polled with a relaxed load; an acquire (which also drops the SM's L1 lines, and
+                // with them the cached hot rows of every block on this SM) is paid once per action, before
+                // the first tile of an action published after this block's last acquire.
+                unsigned tail = (unsigned)ld_relaxed((const int *)&q->tail);
                 if (cur < tail) {
+                    if (cur >= acquired) {
+                        tail = ld_acquire(&q->tail);
+                        acquired = tail;
+                    }
                     BlsAct *e = &q->act[cur];
                     const int n = e->n_tiles;
                     int t = n;
@@ -113,6 +122,7 @@ __device__ __forceinline__ void ring_worker(const BlsParams &p, const RingArgs &
             }
             s_q = got;
             s_tile = tile;
+            s_ctr = 0;
         }
         __syncthreads();
         const int qi = s_q;
@@ -126,13 +136,22 @@ __device__ __forceinline__ void ring_worker(const BlsParams &p, const RingArgs &
             } else if (kind == BLS_ACT_TW_COPY) {
                 tw_copy_tile<8>(p, TileGiven{tile, (unsigned)rank});
             } else if (kind == BLS_ACT_GATHER_TW) {
-                const int run = (int)tile * RPT + warp * GPW + g;      // among the owner's runs, pair-major
-                if (run < e->aux) {
-                    const int chunk = run / a.rpc;                     // (pair of the owner, requester)
-                    const int s0 = (run - chunk * a.rpc) * a.R;
-                    const int i = e->first + chunk / p.P, src = chunk % p.P;
-                    const BlsPairDesc pr = p.pair[i];
-                    stream_run<LANES, DT, 4, false>(p, pr, i, e->slot, src, s0, min(a.R, p.b - s0), lane, nullptr);
+                // a gather tile is RING_GATHER_CHUNK warp-sized pieces; the block's warps take them one by one
+                // (runs differ in length: a fixed split would leave warps idle behind the longest)
+                for (;;) {
+                    int piece = 0;
+                    if ((threadIdx.x & 31) == 0) piece = atomicAdd(&s_ctr, 1);
+                    piece = __shfl_sync(0xffffffffu, piece, 0);
+                    if (piece >= RING_GATHER_CHUNK) break;
+                    const int run = (int)tile * RPT + piece * GPW + g;   // among the owner's runs, pair-major
+                    if (run < e->aux) {
+                        const int chunk = run / a.rpc;                   // (pair of the owner, requester)
+                        const int s0 = (run - chunk * a.rpc) * a.R;
+                        const int i = e->first + chunk / p.P, src = chunk % p.P;
+                        const BlsPairDesc pr = p.pair[i];
+                        stream_run<LANES, DT, 4, false>(p, pr, i, e->slot, src, s0, min(a.R, p.b - s0), lane, nullptr);
+                    }
+                    __syncwarp();
                 }
             }
         } else {
@@ -140,8 +159,15 @@ __device__ __forceinline__ void ring_worker(const BlsParams &p, const RingArgs &
             else if (kind == BLS_ACT_RW_SCAN) rw_scan_tile(p, TileGiven{tile, (unsigned)rank});
             else if (kind == BLS_ACT_RW_SCATTER) rw_scatter_tile(p, TileGiven{tile, (unsigned)rank});
             else if (kind == BLS_ACT_GATHER_RW) {
-                const int run = (int)tile * RPT + warp * GPW + g;
-                if (run < e->aux) rowwise_run<LANES, DT>(p, e->slot, run, a.R, a.rpc, lane, g);
+                for (;;) {
+                    int piece = 0;
+                    if ((threadIdx.x & 31) == 0) piece = atomicAdd(&s_ctr, 1);
+                    piece = __shfl_sync(0xffffffffu, piece, 0);
+                    if (piece >= RING_GATHER_CHUNK) break;
+                    const int run = (int)tile * RPT + piece * GPW + g;
+                    if (run < e->aux) rowwise_run<LANES, DT>(p, e->slot, run, a.R, a.rpc, lane, g);
+                    __syncwarp();
+                }
             }
         }
         __syncthreads();                               // the whole tile is done (and s_q, s_tile have been read)
@@ -184,7 +210,7 @@ template <int LANES, int PART>
 __device__ __forceinline__ void ring_scheduler(const BlsParams &p, const RingArgs &a)
 {
     constexpr bool TW = PART == BLS_PART_TABLE_RR;
-    constexpr int RPT = (BLS_ROUTE_TB / 32) * (32 / LANES);
+    constexpr int RPT = RING_GATHER_CHUNK * (32 / LANES);
     BlsDev *d = p.dev;
     BlsQueue *q = p.queue;
     const int r = threadIdx.x;                         // lane = logical rank
@@ -381,7 +407,7 @@ cudaError_t launch_ring(bls_plan_t *pl, RingArgs &a)
     }
     // as many blocks as stay resident together (a cooperative launch: the workers wait for the
     // scheduler), fewer when the iteration has fewer tiles than that
-    constexpr int RPT = (BLS_ROUTE_TB / 32) * (32 / LANES);
+    constexpr int RPT = RING_GATHER_CHUNK * (32 / LANES);
     const long long gather_tiles = ((long long)(PART == BLS_PART_TABLE_RR ? p.NI : p.T) * p.P * a.rpc + RPT - 1) / RPT + p.P;
     const long long route_tiles = (long long)p.NT * p.P;
     long long want = (gather_tiles > route_tiles ? gather_tiles : route_tiles) + 1;

@@ -55,6 +55,10 @@ template <> struct Acc<BLS_F16> {
     __device__ __forceinline__ float4 hi() const { return make_float4(c.x, c.y, d.x, d.y); }
 };
 
+// A lane's share of a pooled vector: 16 bytes for fp32 tables, 32 bytes (two 16-byte stores) for
+// 16-bit tables.  Streaming stores: outputs are not read again by this kernel.  (One 256-bit
+// store per lane, which writes each 32-byte sector once instead of twice, was measured and is
+// no faster: the store path does not limit these kernels.)
 template <int DT>
 __device__ __forceinline__ void flush(float *o, const Acc<DT> &acc)
 {
