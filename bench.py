@@ -167,7 +167,7 @@ def traffic_record(kernel_src: str, workload_name: str):
         return None
     try:
         rec = json.load(open(path))
-        digest = hashlib.sha256(open(kernel_src, "rb").read()).hexdigest()
+        digest = hashlib.sha256(open(kernel_src, "rb").read() + open(kernel_src + "h", "rb").read()).hexdigest()   # .cu + .cuh
         if rec.get("kernel_sha256") != digest:
             return None
         return float(rec["records"][workload_name]["dram_bytes_per_launch"])
@@ -520,6 +520,7 @@ def run_mine(args):
         for r in range(w.P):
             bls.bls_set_stall(plan, r, delta_ns * (2 if r == w.P - 1 else 1))
         straggler = {"delay_us": delta_ns / 1e3, "last_rank_delay_us": 2 * delta_ns / 1e3}
+        loop(0, 3)                                   # warm-up in this mode (the first launch of the ring kernel loads its code)
         n_s = max(10, args.steps // 4)
         u_s = float(sum(Ls[t % nd] for t in range(n_s)))
         for k in ks:
