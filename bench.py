@@ -61,6 +61,8 @@ def parse_args():
     ap.add_argument("--repeats", type=int, default=5,
                     help="repetitions of the timed loop at the headline bound for the mean and 95 %% confidence interval")
     ap.add_argument("--ks", default="", help="comma-separated bounds to time instead of the workload's own")
+    ap.add_argument("--no-delay-leg", action="store_true",
+                    help="skip the short random-delay measurement (bounded lag at work) on the small 8-rank workload")
     ap.add_argument("--stages", action="store_true",
                     help="time the loop with the dense stages of Listing 1/2 around the lookup (bottom MLP, interaction, "
                          "top MLP; random weights): serial, Listing 1's overlap at k = 0, and Listing 2's at k >= 1")
@@ -309,6 +311,63 @@ def device_tables(w, bls, torch):
     return tabs
 
 
+def host_delay_draws(P: int, n: int, span_ns: int, seed: int) -> np.ndarray:
+    """The delays (ns) the device draws for rank r before iteration j: SplitMix64 output for the state
+    seed + ((r << 40) + j + 1) * golden ratio, modulo span + 1 (the counter-based draw of bls_set_random_stall)."""
+    rr = np.arange(P, dtype=np.uint64).reshape(-1, 1)
+    jj = np.arange(n, dtype=np.uint64).reshape(1, -1)
+    with np.errstate(over="ignore"):
+        z = np.uint64(seed) + ((rr << np.uint64(40)) + jj + np.uint64(1)) * np.uint64(0x9E3779B97F4A7C15)
+        z = (z ^ (z >> np.uint64(30))) * np.uint64(0xBF58476D1CE4E5B9)
+        z = (z ^ (z >> np.uint64(27))) * np.uint64(0x94D049BB133111EB)
+        z = z ^ (z >> np.uint64(31))
+    return (z % np.uint64(span_ns + 1)).astype(np.float64)
+
+
+def delay_leg(bls, torch, mean_delay_us=300.0, steps=150):
+    """Bounded lag at work (Section V-E setting 2, Section VI-B), on a small workload of its own: 26 one-hot
+    tables, 8 logical ranks, batch 2048; every rank is delayed by U(0, 2 D) before each of its iterations.
+    Time per step for bounds 0, 1 and 4, with the closed forms beside it."""
+    w = bi.workload(2, 0.05, 1.0)
+    tabs = [torch.from_numpy(bi.table_values(t)).cuda() for t in w.tables]
+    inputs = [bi.make_iteration(w, it) for it in range(8)]
+    d_in = [(torch.from_numpy(i).cuda(), torch.from_numpy(o).cuda()) for i, o in inputs]
+    plan = bls.bls_plan(tabs, w.partition, w.P, w.local_batch, 4, capacity(w, inputs))
+    bls.bls_set_ring(plan, 1)
+
+    def timed(k):
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for t in range(steps):
+            bls.bls_step(plan, k, *d_in[t % 8])
+        while bls.bls_drain(plan)[0] is not None:
+            pass
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / steps * 1e3
+
+    timed(0)
+    work_us = timed(0)
+    span_ns = int(2 * mean_delay_us * 1000)
+    for r in range(w.P):
+        bls.bls_set_random_stall(plan, r, span_ns, 7)
+    out = {"workload": w.name, "ranks": w.P, "mean_delay_us": mean_delay_us, "steps": steps, "work_us": work_us,
+           "closed_form_k0_us": work_us + 2 * mean_delay_us * w.P / (w.P + 1), "closed_form_k_inf_us": work_us + mean_delay_us}
+    first = 2 * steps
+    for k in (0, 1, 4):
+        us = timed(k)
+        done = bls.bls_timeline(plan, first, steps)[2].astype(np.int64)
+        first += steps
+        lat = np.diff(done, axis=0).mean(axis=0) / 1e3
+        out[f"k{k}_us_per_step"] = us
+        out[f"k{k}_throughput_batches_per_s"] = float(np.sum(1e6 / lat))     # Section V-C: T = sum over ranks of batches / L
+    st, lag = bls.bls_status(plan)
+    out["max_lag"], out["status"] = lag, st
+    out["hidden_by_k1"] = (out["k0_us_per_step"] - out["k1_us_per_step"]) / max(1e-9, out["k0_us_per_step"] - out["closed_form_k_inf_us"])
+    return out
+
+
 def plan_iterations(bls, plan) -> int:
     """Iterations the plan has issued so far (all ranks agree between loops)."""
     return int(bls.bls_counters(plan)[0][0])
@@ -481,14 +540,7 @@ def run_mine(args):
         from oracle.ring_model import makespan       # the timing model is test infrastructure: reported beside, never used
         span_ns, seed = int(2 * args.delay_us * 1000), 2024
         n_d = min(args.steps, 1000)
-        rr = np.arange(w.P, dtype=np.uint64).reshape(-1, 1)
-        jj = np.arange(n_d, dtype=np.uint64).reshape(1, -1)
-        with np.errstate(over="ignore"):
-            z = np.uint64(seed) + ((rr << np.uint64(40)) + jj + np.uint64(1)) * np.uint64(0x9E3779B97F4A7C15)
-            z = (z ^ (z >> np.uint64(30))) * np.uint64(0xBF58476D1CE4E5B9)
-            z = (z ^ (z >> np.uint64(27))) * np.uint64(0x94D049BB133111EB)
-            z = z ^ (z >> np.uint64(31))
-        delays_us = (z % np.uint64(span_ns + 1)).astype(np.float64) / 1e3
+        delays_us = host_delay_draws(w.P, n_d, span_ns, seed) / 1e3
         # stall-free time per step in the same mode (ring kernel), the model's per-iteration work
         bls.bls_set_ring(plan, 1)
         loop(0, 5)
@@ -528,6 +580,18 @@ def run_mine(args):
             straggler[str(k)] = {"ms_per_step": ms / n_s}
         for r in range(w.P):
             bls.bls_set_stall(plan, r, 0)
+    # the paper's per-process metrics (Section V-C) for a loop at the headline bound, from the device's time stamps
+    first_it = plan_iterations(bls, plan)
+    n_tl = min(args.steps, 1000)
+    loop(k_head, n_tl)
+    done_ns = bls.bls_timeline(plan, first_it, n_tl)[2].astype(np.int64)
+    lat_ms = np.diff(done_ns, axis=0).mean(axis=0) / 1e6 if n_tl > 1 else np.zeros(w.P)
+    paper_metrics = {"latency_ms_per_batch_per_rank": {"min": float(lat_ms.min()), "max": float(lat_ms.max())},
+                     "throughput_batches_per_s": float(np.sum(1e3 / lat_ms)) if n_tl > 1 else None,
+                     "note": "L = mean time between a logical rank's consecutive completions, T = sum over ranks of 1 / L"}
+    bounded_lag = None
+    if rank == 0 and not args.no_delay_leg:
+        bounded_lag = delay_leg(bls, torch)
     clocks = sampler.stop() if sampler else None
     st, lag = bls.bls_status(plan)
     if st != bls.BLS_OK:
@@ -579,6 +643,7 @@ def run_mine(args):
         "stage_ms_per_step": {"route": prof["ms_route"] / max(1, prof["calls"]), "gather_pool_return": ms_gather,
                               "ring": prof["ms_ring"] / max(1, prof["calls"])},
         "clocks": clocks, "e2e": e2e, "gpu_launches": launches, "delay_sweep": delay_sweep, "straggler": straggler,
+        "paper_metrics": paper_metrics, "bounded_lag_with_random_delays": bounded_lag,
     }
     if not args.no_cpu_baseline and world == 1:
         result["cpu_baseline"], result["parity"] = cpu_baseline(w, inputs, gpu_out0)
