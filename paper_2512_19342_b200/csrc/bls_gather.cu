@@ -242,11 +242,7 @@ static void launch_gather(const bls_plan_t *pl)
             const bool deep = pl->rows_in_flight >= 32;
             const size_t smem = (size_t)(4 * (32 / LANES)) * ((deep ? 4 : 2) * BR * LANES * 16 + (deep ? 4 : 2) * 8);
             auto kernel = deep ? bls_gather_bulk_kernel<LANES, DT, BR, 4> : bls_gather_bulk_kernel<LANES, DT, BR, 2>;
-            static size_t configured[2] = {0, 0};
-            if (configured[deep] != smem) {
-                cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-                configured[deep] = smem;
-            }
+            cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);   // per device, cheap: every launch
             int per = 1;
             cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per, kernel, 128, smem);
             const long long want2 = (n_runs + 4 * (32 / LANES) - 1) / (4 * (32 / LANES));

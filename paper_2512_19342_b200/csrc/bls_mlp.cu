@@ -356,12 +356,9 @@ template <int BN>
 cudaError_t launch_linear_bn(const CUtensorMap &mx, const CUtensorMap &mw, const LinArgs &a, cudaStream_t s)
 {
     const size_t smem = 1024 + (size_t)MLP_STAGES * (MLP_BM + BN) * MLP_BK * 2;
-    static bool configured = false;
-    if (!configured) {
-        cudaError_t e = cudaFuncSetAttribute(bls_linear_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-        if (e != cudaSuccess) return e;
-        configured = true;
-    }
+    // set on every launch: the attribute belongs to the current device, and the call costs about a microsecond
+    cudaError_t e = cudaFuncSetAttribute(bls_linear_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
     dim3 grid((a.N + BN - 1) / BN, (a.M + MLP_BM - 1) / MLP_BM);
     bls_linear_kernel<BN><<<grid, MLP_THREADS, smem, s>>>(mx, mw, a);
     return cudaGetLastError();

@@ -369,6 +369,60 @@ def test_constant_straggler_is_not_masked_but_costs_nothing_extra():
     assert times[1] <= times[0] * 1.01 and times[4] <= times[0] * 1.01, times
 
 
+def test_ring_kernel_corner_shapes():
+    """The persistent ring kernel on shapes at the edges: a single logical rank; more ranks than tables
+    (owners without tables answer at once); host-buffer entry points; hot-row staging switched on (the
+    ring kernel gathers without it, the router still marks the lookups)."""
+    for w in (bi.tiny_workload(T=4, P=1, b=300, rows=1000, dim=32, lengths="poisson20c"),
+              bi.tiny_workload(T=2, P=5, b=3, rows=50, dim=8),
+              bi.tiny_workload(T=3, P=4, b=50, rows=300, dim=32, dtype="f16", partition="row_block", lengths="extremes")):
+        data = [bi.table_values(t) for t in w.tables]
+        tabs = dev_tables(w, data)
+        outs, inputs, status, lag = run_loop(w, tabs, 2, 6, ring=1, stalls={0: 150_000})
+        assert status == bls.BLS_OK and lag <= 2
+        assert_matches_oracle(w, data, inputs, outs)
+    # host buffers in, host vectors out, with a delayed rank
+    w = bi.workload(3, 0.01, 0.02)
+    data = [bi.table_values(t) for t in w.tables]
+    tabs = dev_tables(w, data)
+    plan = make_plan(w, tabs, 2)
+    bls.bls_set_stall(plan, 3, 200_000)
+    host_out = torch.empty(w.P, w.local_batch, w.T, w.tables[0].dim, dtype=torch.float32).pin_memory()
+    got, inputs = {}, [bi.make_iteration(w, t) for t in range(5)]
+    for ids, off in inputs:
+        it = bls.bls_step_host(plan, 2, torch.from_numpy(ids).pin_memory(), torch.from_numpy(off).pin_memory(), host_out)
+        torch.cuda.synchronize()
+        if it >= 0:
+            got[it] = host_out.clone()
+    while True:
+        it = bls.bls_drain_host(plan, host_out)
+        torch.cuda.synchronize()
+        if it < 0:
+            break
+        got[it] = host_out.clone()
+    assert sorted(got) == list(range(5)) and bls.bls_status(plan)[0] == bls.BLS_OK
+    assert_matches_oracle(w, data, inputs, got)
+    # hot-row staging attached and built, then a delay: the loop goes on in the ring kernel
+    plan = make_plan(w, tabs, 1)
+    bls.bls_hot_attach(plan, 64)
+    for ids, off in inputs[:2]:
+        bls.bls_hot_observe(plan, torch.from_numpy(ids).cuda(), torch.from_numpy(off).cuda())
+    bls.bls_hot_build(plan)
+    bls.bls_set_stall(plan, 1, 100_000)
+    outs = []
+    for ids, off in inputs:
+        out, it = bls.bls_step(plan, 1, torch.from_numpy(ids).cuda(), torch.from_numpy(off).cuda())
+        if out is not None:
+            outs.append(out.clone())
+    while True:
+        out, it = bls.bls_drain(plan)
+        if out is None:
+            break
+        outs.append(out.clone())
+    assert bls.bls_status(plan)[0] == bls.BLS_OK
+    assert_matches_oracle(w, data, inputs, outs)
+
+
 def test_largest_ring():
     """k_max = 15 (16 slots) and 32 ranks, the limits of a plan."""
     w = bi.tiny_workload(T=6, P=32, b=3, rows=50, dim=8, lengths="mixed")

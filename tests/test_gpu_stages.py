@@ -144,3 +144,25 @@ def test_lookup_and_stages_end_to_end():
         want = stages.mlp(r_want, tw, tb, "none")
         err = oracle.vector_rel_err(got[t].astype(np.float64), want)
         assert err <= 1e-2, (t, err)
+
+
+def test_stage_calls_reject_bad_arguments():
+    """Argument checks of the dense-stage entry points happen on the host, before any GPU work."""
+    import ctypes as C
+    lib = bls.lib()
+    n = C.c_size_t(0)
+    dims = (C.c_int * 3)(16, 12, 8)                          # a hidden width that is not a multiple of 8
+    assert lib.bls_mlp_bytes(2, dims, 128, C.byref(n)) == bls.BLS_EINVAL
+    dims = (C.c_int * 3)(16, 64, 8)
+    assert lib.bls_mlp_bytes(2, dims, 0, C.byref(n)) == bls.BLS_EINVAL
+    assert lib.bls_mlp_bytes(2, dims, 128, C.byref(n)) == bls.BLS_OK and n.value >= 128 * 64 * 2
+    rng = np.random.Generator(np.random.PCG64(0))
+    mlp, _, _ = make_mlp(rng, [16, 64, 8], 1, 128)
+    x = torch.zeros(200, 16, dtype=torch.bfloat16, device="cuda")
+    y = torch.zeros(200, 8, dtype=torch.bfloat16, device="cuda")
+    with pytest.raises(bls.BlsError) as e:
+        mlp.forward(x, y)                                    # more rows than the handle was made for
+    assert e.value.code == bls.BLS_EINVAL
+    with pytest.raises(bls.BlsError):
+        bls.bls_interact(x, torch.zeros(200, 3, 16, device="cuda"), torch.zeros(200, 16, dtype=torch.bfloat16, device="cuda"))   # r too narrow
+    assert torch.ones(4, device="cuda").sum().item() == 4.0
