@@ -181,6 +181,30 @@ def test_delays_switched_on_and_off_mid_flight():
     assert posted == served == done == [n_iter] * w.P
 
 
+def test_ring_mode_and_timeline_call_rules():
+    """bls_set_ring only between loops; bls_timeline only for iterations that have been issued."""
+    w = bi.workload(1)
+    tabs = dev_tables(w, [bi.table_values(t) for t in w.tables])
+    plan = make_plan(w, tabs, 2)
+    ids, off = bi.make_iteration(w, 0)
+    d_ids, d_off = torch.from_numpy(ids).cuda(), torch.from_numpy(off).cuda()
+    with pytest.raises(bls.BlsError) as e:
+        bls.bls_timeline(plan, 0, 1)                              # nothing issued yet
+    assert e.value.code == bls.BLS_ESTATE
+    bls.bls_set_ring(plan, 1)
+    bls.bls_step(plan, 2, d_ids, d_off)
+    with pytest.raises(bls.BlsError) as e:
+        bls.bls_set_ring(plan, -1)                                # an iteration is outstanding
+    assert e.value.code == bls.BLS_ESTATE
+    while bls.bls_drain(plan)[0] is not None:
+        pass
+    bls.bls_set_ring(plan, -1)
+    post, serve, done = bls.bls_timeline(plan, 0, 1)
+    assert post.shape == (1, w.P) and np.all(post > 0) and np.all(serve >= post.max()) and np.all(done >= serve.max())
+    with pytest.raises(bls.BlsError):
+        bls.bls_timeline(plan, 0, 2)                              # iteration 1 does not exist
+
+
 def test_changing_k_mid_flight_is_refused():
     w = bi.workload(1)
     tabs = dev_tables(w, [bi.table_values(t) for t in w.tables])
