@@ -141,6 +141,9 @@ bls_linear_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
     const int nkb = (a.K + MLP_BK - 1) / MLP_BK;
 
     if (threadIdx.x == 0) {
+        // fetch the two tensor maps now: the first tile loads would otherwise wait for them
+        asm volatile("prefetch.tensormap [%0];" ::"l"(&map_x) : "memory");
+        asm volatile("prefetch.tensormap [%0];" ::"l"(&map_w) : "memory");
         for (int s = 0; s < MLP_STAGES; s++) { mb_init(full0 + 8 * s, 1); mb_init(empty0 + 8 * s, 1); }
         mb_init(done_bar, 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
