@@ -320,6 +320,7 @@ static void enqueue_wave(bls_plan_t *pl, int mode, long long t_last, long long f
     bls_launch_gate(pl, mode, t_last, floor_, k, ids, off, n_ids);
     bls_launch_route(pl);
     if (ev) cudaEventRecord(ev[1], pl->stream);
+    pl->serve_n_ids = pl->n_ids_of[t_last % pl->prm.S];   // without delays a wave answers the newest iteration
     bls_launch_gather(pl);                             // its last block commits the wave
     if (ev) { cudaEventRecord(ev[2], pl->stream); cudaEventRecord(ev[3], pl->stream); }
     pl->kernels_launched += 2 + bls_route_kernels(pl);
@@ -356,6 +357,7 @@ static void enqueue_wave_overlapped(bls_plan_t *pl, long long t_last, long long 
     bls_launch_gate(pl, BLS_MODE_STEP, t_last, floor_, k, ids, off, n_ids, 1);
     cudaEventRecord(pl->e_fork, pl->stream);
     if (ev) cudaEventRecord(ev[1], pl->stream);
+    pl->serve_n_ids = t_last >= 1 ? pl->n_ids_of[(t_last - 1) % pl->prm.S] : -1;   // the owners answer iteration t - 1
     bls_launch_gather(pl);                             // first, so that its blocks are resident first
     cudaStreamWaitEvent(pl->s_side, pl->e_fork, 0);
     bls_launch_meta(pl, pl->s_side);                   // chunk bases, send counts and displacements of iteration t
@@ -414,6 +416,7 @@ bls_status_t bls_route(bls_plan_t *pl, int64_t iter, const int32_t *ids, const i
     if (!pl || !offsets || (!ids && n_ids > 0) || n_ids < 0) return BLS_EINVAL;
     if (iter != pl->t_next || pl->t_handed != pl->t_next || pl->routed_only >= 0) return BLS_ESTATE;
     poison_slot(pl, iter);
+    pl->n_ids_of[iter % pl->prm.S] = n_ids;
     bls_launch_gate(pl, BLS_MODE_ROUTE_ONLY, iter, -1, 0, ids, offsets, n_ids);
     bls_launch_route(pl);
     bls_launch_commit(pl);
@@ -428,6 +431,7 @@ bls_status_t bls_lookup(bls_plan_t *pl, int64_t iter)
     if (!pl) return BLS_EINVAL;
     if (pl->routed_only != iter) return BLS_ESTATE;
     bls_launch_gate(pl, BLS_MODE_LOOKUP_ONLY, iter, -1, 0, nullptr, nullptr, 0);
+    pl->serve_n_ids = pl->n_ids_of[iter % pl->prm.S];
     bls_launch_gather(pl);                             // its last block commits the wave
     pl->kernels_launched += 2;
     pl->routed_only = -1;
@@ -444,6 +448,7 @@ bls_status_t bls_step(bls_plan_t *pl, int k, const int32_t *ids, const int32_t *
     pl->k_cur = k;
     const long long t = pl->t_next++;
     poison_slot(pl, t);
+    pl->n_ids_of[t % pl->prm.S] = n_ids;
     // (iterations below about a million lookups are bound by the launch rate, of the host or of
     // the GPU, and the second stream costs five more driver calls per step: they stay on one stream)
     const bool ring = ring_applies(pl);

@@ -41,15 +41,17 @@ __device__ __forceinline__ void tw_copy_tile(const BlsParams &p, const Where whe
     const int cn = cbp[i + 1] - cb;              // chunk length accepted by the meta kernel
     const long long off0 = c.off[g0];
     __shared__ int s_lo, s_hi;
+    bool other_length = false;                   // a bag that does not hold exactly one ID
     for (int s = threadIdx.x; s < nb; s += blockDim.x) {
         int st, en;
         if (!bag_range(c, g0 + s0 + s, off0, cn, st, en)) flag(p, BLS_ST_EINVAL);
+        other_length |= en - st != 1;
         int pos = cb + st;
         c.sub_start[(size_t)i * p.b + s0 + s] = pos > p.cap ? p.cap : pos;
         if (s == 0) s_lo = st;
         if (s == nb - 1) s_hi = en;
     }
-    __syncthreads();
+    if (__syncthreads_or(other_length) && threadIdx.x == 0) p.dev->onehot[c.slot] = 0;   // (the barrier also publishes s_lo, s_hi)
     const unsigned rows = (unsigned)p.tab[t].rows;
     const int lo = s_lo, hi = max(s_lo, s_hi);
     const int *in = c.ids + off0;
