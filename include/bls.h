@@ -215,7 +215,12 @@ bls_status_t bls_set_overlap(bls_plan_t *plan, int mode);
  * with 0xFF bytes (NaN), so that a bag that was not written, or a slot read before its data
  * arrived, shows up in the result.  Costs one pass over the slot per step. */
 bls_status_t bls_set_poison(bls_plan_t *plan, int enable);
-/* Upper limit of any single device-side wait (default 2 s). */
+/* Upper limit of any single device-side wait (default 2 s).  In the ring kernel: after this long
+ * without any progress (no rank changed state, no tile of work finished) the scheduler latches
+ * BLS_ETIMEOUT and stops honouring injected delays, so the loop still completes with correct data;
+ * after a second such period it ends the launch.  A worker block that finds no work for four
+ * times the limit plus one second leaves.  Waits on mbarriers (bulk-copy gather variant, linear
+ * layers) give up after 2 s of their own. */
 bls_status_t bls_set_wait_limit(bls_plan_t *plan, int64_t ns);
 
 /* Stage timing with CUDA events on the plan's stream.  While enabled, every
@@ -224,7 +229,8 @@ bls_status_t bls_set_wait_limit(bls_plan_t *plan, int64_t ns);
  * calls into milliseconds per stage (gate + router kernels, the gather-pool-return
  * kernel including the commit done by its last block, anything after it), reports how
  * many calls were summed and how many kernels the plan has launched so far, and clears
- * the record.  Any pointer may be NULL. */
+ * the record.  Any pointer may be NULL.  A call served by the ring kernel is one launch: its
+ * whole time is reported under the gather stage. */
 bls_status_t bls_profile(bls_plan_t *plan, int enable);
 bls_status_t bls_profile_read(bls_plan_t *plan, double *ms_route, double *ms_gather, double *ms_ring,
                               int64_t *calls, int64_t *kernels);
