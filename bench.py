@@ -591,7 +591,10 @@ def run_mine(args):
                      "note": "L = mean time between a logical rank's consecutive completions, T = sum over ranks of 1 / L"}
     bounded_lag = None
     if rank == 0 and not args.no_delay_leg:
-        bounded_lag = delay_leg(bls, torch)
+        try:                                          # an extra leg: its failure must not cost the benchmark line
+            bounded_lag = delay_leg(bls, torch)
+        except Exception as exc:                      # noqa: BLE001
+            bounded_lag = {"error": f"{type(exc).__name__}: {exc}"}
     clocks = sampler.stop() if sampler else None
     st, lag = bls.bls_status(plan)
     if st != bls.BLS_OK:
