@@ -69,6 +69,9 @@ def parse_args():
     ap.add_argument("--ring", type=int, default=None, choices=[-1, 0, 1],
                     help="persistent ring kernel: -1 only with injected delays, 0 also for small iterations, 1 always "
                          "(default: the library's own choice)")
+    ap.add_argument("--fused", type=int, default=None, choices=[-1, 0, 1],
+                    help="one-launch kernel for small table-wise iterations: -1 never, 0 by iteration size, 1 whenever "
+                         "it applies (default: the library's own choice)")
     return ap.parse_args()
 
 
@@ -414,6 +417,8 @@ def run_mine(args):
         bls.bls_set_tuning(plan, *[int(x) for x in args.tune.split(",")])
     if args.ring is not None:
         bls.bls_set_ring(plan, args.ring)
+    if args.fused is not None:
+        bls.bls_set_fused(plan, args.fused)
     hot_k = HOT_DEFAULT.get(args.config, 0) if args.hot < 0 else args.hot
     if hot_k and w.partition == "table_rr":
         # request statistics come from two batches that are not among the timed ones
@@ -608,6 +613,12 @@ def run_mine(args):
     L_mean = float(np.mean(Ls))
     step_bytes, gather_bytes = algorithmic_bytes(w, L_mean)
     ms_gather = prof["ms_gather"] / max(1, prof["calls"])
+    one_launch = launches == args.steps and w.partition == "table_rr" and not args.ring
+    if one_launch:
+        # small iterations: the library ran every step as ONE launch (bls_small_tw_kernel), which does the whole
+        # step; its duration is the time per step of the timed loop (events around each launch would cost as much
+        # as the launch)
+        gather_kernel, gather_bytes, ms_gather = "bls_small_tw_kernel", step_bytes, ms_head / args.steps
     ach = gather_bytes / (ms_gather * 1e-3) / 1e9
     traffic = traffic_record(os.path.join(ROOT, "paper_2512_19342_b200", "csrc", "bls_gather.cu"), w.name)
     dram_gbs = None if traffic is None else traffic / (ms_gather * 1e-3) / 1e9
@@ -643,7 +654,8 @@ def run_mine(args):
             "note": "same kernel and bag lengths, IDs drawn uniformly: every row read goes to DRAM, so this is the "
                     "kernel's DRAM-bound figure; with the workload's Zipf IDs hot rows hit L1/L2 and roofline.frac "
                     "exceeds 1 while roofline.traffic (DRAM bytes) stays far below the algorithmic bytes"},
-        "stage_ms_per_step": {"route": prof["ms_route"] / max(1, prof["calls"]), "gather_pool_return": ms_gather,
+        "stage_ms_per_step": {"route": prof["ms_route"] / max(1, prof["calls"]),
+                              "gather_pool_return": prof["ms_gather"] / max(1, prof["calls"]),
                               "ring": prof["ms_ring"] / max(1, prof["calls"])},
         "clocks": clocks, "e2e": e2e, "gpu_launches": launches, "delay_sweep": delay_sweep, "straggler": straggler,
         "paper_metrics": paper_metrics, "bounded_lag_with_random_delays": bounded_lag,

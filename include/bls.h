@@ -132,7 +132,8 @@ bls_status_t bls_lookup(bls_plan_t *plan, int64_t iter);
  *           every rank (the oldest request is waited for once more than k are
  *           outstanding) and hands it back: *out = its fp32 [P][b][T][dim] block
  *           inside the ring, *out_iter = t-k; or *out = NULL, *out_iter = -1
- *           while t < k.  `*out` stays valid until the next bls_step/bls_drain
+ *           during the first k steps of a loop (iteration t-k does not exist, or belongs
+ *           to an earlier loop that has been drained).  `*out` stays valid until the next bls_step/bls_drain
  *           call on the stream.  ids/offsets of iteration t are borrowed until
  *           k further steps (or the drain) have run.
  *           With k >= 1, table-wise placement, no injected delays and iterations of about
@@ -145,6 +146,10 @@ bls_status_t bls_lookup(bls_plan_t *plan, int64_t iter);
  *           iteration behind the requesters after a step (bls_status reports a lag of 1)
  *           and the first bls_drain call enqueues the last answer.  Results are the same
  *           bit for bit in both modes.
+ *           Small table-wise iterations without injected delays (below about 256 K lookups;
+ *           bls_set_fused) are ONE kernel launch: every block routes a tile of one
+ *           (requester, table) chunk and answers it at once, the last block publishes the
+ *           iteration for all ranks.  Same routing artefacts, same sums, bit for bit.
  * bls_drain: Listing 2's final loop, one outstanding iteration per call, oldest
  *           first; *out = NULL once nothing is outstanding. */
 bls_status_t bls_step(bls_plan_t *plan, int k, const int32_t *ids, const int32_t *offsets,
@@ -164,7 +169,7 @@ bls_status_t bls_step_host(bls_plan_t *plan, int k, const int32_t *ids /*host*/,
 bls_status_t bls_drain_host(bls_plan_t *plan, float *host_out /*host*/, int64_t *out_iter /*host out*/);
 
 /* ---- inspection (bls_view, bls_counters, bls_status, bls_set_poison, bls_set_wait_limit,
- * bls_profile*, bls_set_tuning, bls_set_overlap, bls_set_ring: debugging and measurement aids with no counterpart in the paper) ---- */
+ * bls_profile*, bls_set_tuning, bls_set_overlap, bls_set_fused, bls_set_ring: debugging and measurement aids with no counterpart in the paper) ---- */
 /* Device pointers of the slot that holds iteration `iter` (must still be in the ring). */
 bls_status_t bls_view(bls_plan_t *plan, int64_t iter, bls_route_view_t *view /*host out*/);
 /* Synchronises the stream; copies the P per-rank counters to host arrays (may be NULL). */
@@ -211,6 +216,12 @@ bls_status_t bls_timeline(bls_plan_t *plan, int64_t first_iter, int n_iter, uint
  * table-wise placement, no injected delays, no hot-row staging, ring kernel not in use), -1 never.
  * May be called at any time. */
 bls_status_t bls_set_overlap(bls_plan_t *plan, int mode);
+/* One-launch iterations (see bls_step): mode 0 (default) uses the fused kernel when an iteration
+ * holds fewer than about 256 K lookups (P * max_ids_per_rank < 2^18: below that the launches of a
+ * wave cost more than the work in them), 1 whenever it applies (table-wise placement, no injected
+ * delays, ring kernel and overlapped mode not in use, no hot-row staging, default tuning), -1 never.
+ * May be called at any time. */
+bls_status_t bls_set_fused(bls_plan_t *plan, int mode);
 /* Debug aid: while enabled, the output slot an iteration is issued into is first filled
  * with 0xFF bytes (NaN), so that a bag that was not written, or a slot read before its data
  * arrived, shows up in the result.  Costs one pass over the slot per step. */

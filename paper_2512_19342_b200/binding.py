@@ -6,6 +6,7 @@ no CPU fallback: if the shared library is missing the first call raises.
 """
 from __future__ import annotations
 
+import collections
 import ctypes as C
 import os
 from typing import List, Optional, Sequence, Tuple
@@ -25,7 +26,7 @@ EXPORTS = ["bls_plan_bytes", "bls_plan", "bls_destroy", "bls_route", "bls_lookup
            "bls_drain", "bls_step_host", "bls_drain_host", "bls_view", "bls_counters", "bls_status",
            "bls_set_stall", "bls_set_wait_limit", "bls_strerror", "bls_fill_hash_table",
            "bls_profile", "bls_profile_read", "bls_set_tuning", "bls_route_table_rr_static",
-           "bls_set_random_stall", "bls_set_ring", "bls_timeline", "bls_set_poison", "bls_set_overlap", "bls_a2a_bytes", "bls_a2a_create", "bls_a2a_destroy", "bls_a2a_post", "bls_a2a_wait",
+           "bls_set_random_stall", "bls_set_ring", "bls_timeline", "bls_set_poison", "bls_set_overlap", "bls_set_fused", "bls_a2a_bytes", "bls_a2a_create", "bls_a2a_destroy", "bls_a2a_post", "bls_a2a_wait",
            "bls_a2a_status", "bls_mlp_bytes", "bls_mlp_create", "bls_mlp_destroy", "bls_mlp_forward", "bls_interact",
            "bls_mlp_status", "bls_hot_bytes", "bls_hot_attach", "bls_hot_observe", "bls_hot_build", "bls_hot_view"]
 
@@ -60,6 +61,8 @@ def lib():
         _lib = C.CDLL(LIB_PATH)
         _lib.bls_strerror.restype = C.c_char_p
         _lib.bls_strerror.argtypes = [C.c_int]
+        # the call of the inner loop: with declared argument types plain Python integers can be passed
+        _lib.bls_step.argtypes = [C.c_void_p, C.c_int, C.c_void_p, C.c_void_p, C.c_int64, C.c_void_p, C.c_void_p]
     return _lib
 
 
@@ -89,11 +92,12 @@ class Plan:
         self.handle, self.tables, self.workspace = handle, list(tables), workspace
         self.P, self.T, self.b, self.D, self.k_max, self.part = P, T, b, D, k_max, part
         self.stream = stream
-        self._borrowed: List[Tuple[torch.Tensor, torch.Tensor]] = []
-
-    def _keep(self, ids, offsets):
-        self._borrowed.append((ids, offsets))
-        del self._borrowed[:-(self.k_max + 2)]
+        # inputs of the iterations still in the ring stay referenced here (the library borrows them)
+        self._borrowed = collections.deque(maxlen=k_max + 2)
+        self._keep = self._borrowed.append
+        self._outs = {}                      # output slot address -> tensor view (a ring has k_max + 1 of them)
+        self._ret = (C.c_void_p(), C.c_int64(-1))   # bls_step / bls_drain write their results here
+        self._ret_refs = (C.byref(self._ret[0]), C.byref(self._ret[1]))
 
     def _wrap(self, ptr: int, n_elems: int, dtype: torch.dtype) -> torch.Tensor:
         off = ptr - self.workspace.data_ptr()
@@ -101,7 +105,11 @@ class Plan:
         return self.workspace[off:off + nbytes].view(dtype)
 
     def out_tensor(self, ptr: int) -> torch.Tensor:
-        return self._wrap(ptr, self.P * self.b * self.T * self.D, torch.float32).view(self.P, self.b, self.T, self.D)
+        t = self._outs.get(ptr)
+        if t is None:
+            t = self._wrap(ptr, self.P * self.b * self.T * self.D, torch.float32).view(self.P, self.b, self.T, self.D)
+            self._outs[ptr] = t
+        return t
 
     def __del__(self):
         h, self.handle = getattr(self, "handle", None), None
@@ -136,7 +144,7 @@ def bls_plan(tables: Sequence[torch.Tensor], part: str, P: int, local_batch: int
 
 
 def bls_route(plan: Plan, it: int, ids: torch.Tensor, offsets: torch.Tensor) -> None:
-    plan._keep(ids, offsets)
+    plan._keep((ids, offsets))
     _check(lib().bls_route(plan.handle, C.c_int64(it), C.c_void_p(ids.data_ptr()),
                            C.c_void_p(offsets.data_ptr()), C.c_int64(ids.numel())), "bls_route")
 
@@ -147,23 +155,24 @@ def bls_lookup(plan: Plan, it: int) -> None:
 
 def bls_step(plan: Plan, k: int, ids: torch.Tensor, offsets: torch.Tensor):
     """Returns (out, out_iter): out is a [P][b][T][D] fp32 view into the ring or None."""
-    plan._keep(ids, offsets)
-    out, it = C.c_void_p(), C.c_int64(-1)
-    _check(lib().bls_step(plan.handle, k, C.c_void_p(ids.data_ptr()), C.c_void_p(offsets.data_ptr()),
-                          C.c_int64(ids.numel()), C.byref(out), C.byref(it)), "bls_step")
+    plan._keep((ids, offsets))
+    (out, it), (p_out, p_it) = plan._ret, plan._ret_refs
+    code = lib().bls_step(plan.handle, k, ids.data_ptr(), offsets.data_ptr(), ids.numel(), p_out, p_it)
+    if code != BLS_OK:
+        raise BlsError(code, "bls_step")
     return (plan.out_tensor(out.value) if out.value else None), it.value
 
 
 def bls_drain(plan: Plan):
-    out, it = C.c_void_p(), C.c_int64(-1)
-    _check(lib().bls_drain(plan.handle, C.byref(out), C.byref(it)), "bls_drain")
+    (out, it), (p_out, p_it) = plan._ret, plan._ret_refs
+    _check(lib().bls_drain(plan.handle, p_out, p_it), "bls_drain")
     return (plan.out_tensor(out.value) if out.value else None), it.value
 
 
 def bls_step_host(plan: Plan, k: int, ids: torch.Tensor, offsets: torch.Tensor,
                   host_out: Optional[torch.Tensor]) -> int:
     """ids/offsets/host_out are HOST tensors (pinned recommended); returns the iteration copied out or -1."""
-    plan._keep(ids, offsets)
+    plan._keep((ids, offsets))
     it = C.c_int64(-1)
     _check(lib().bls_step_host(plan.handle, k, C.c_void_p(ids.data_ptr()), C.c_void_p(offsets.data_ptr()),
                                C.c_int64(ids.numel()),
@@ -235,6 +244,11 @@ def bls_set_poison(plan: Plan, enable: bool) -> None:
 def bls_set_overlap(plan: Plan, mode: int) -> None:
     """-1 never, 0 by iteration size (default), 1 whenever the overlapped mode applies."""
     _check(lib().bls_set_overlap(plan.handle, int(mode)), "bls_set_overlap")
+
+
+def bls_set_fused(plan: Plan, mode: int) -> None:
+    """One-launch kernel for small table-wise iterations: -1 never, 0 by iteration size (default), 1 whenever it applies."""
+    _check(lib().bls_set_fused(plan.handle, int(mode)), "bls_set_fused")
 
 
 def bls_set_wait_limit(plan: Plan, ns: int) -> None:

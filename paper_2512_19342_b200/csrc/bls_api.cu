@@ -381,6 +381,27 @@ static bool ring_applies(const bls_plan_t *pl)
            (long long)pl->prm.P * pl->prm.cap < (1 << 17);
 }
 
+// Small table-wise iterations with the ranks in lockstep: the whole iteration in one launch
+// (bls_small.cu).  Measured against the wave of stand-alone kernels it is 2.5 times faster at
+// 50 K lookups per iteration, 1.7 times at 200 K, and level from about 350 K (20-ID bags) to
+// 1 M (one-ID bags) lookups.
+static bool small_applies(const bls_plan_t *pl)
+{
+    const BlsParams &p = pl->prm;
+    if (pl->fused_mode < 0 || p.part != BLS_PART_TABLE_RR || p.hot.enabled || pl->rows_in_flight != 4) return false;
+    return pl->fused_mode > 0 || (long long)p.P * p.cap < (1 << 18);
+}
+
+static void enqueue_small(bls_plan_t *pl, long long t, const int *ids, const int *off, long long n_ids)
+{
+    cudaEvent_t *ev = nullptr;
+    if (pl->prof_on && pl->prof_n < BLS_PROF_MAX && pl->prof_ev) ev = pl->prof_ev + (size_t)pl->prof_n++ * 4;
+    if (ev) { cudaEventRecord(ev[0], pl->stream); cudaEventRecord(ev[1], pl->stream); }
+    bls_launch_small(pl, t, ids, off, n_ids);
+    if (ev) { cudaEventRecord(ev[2], pl->stream); cudaEventRecord(ev[3], pl->stream); }
+    pl->kernels_launched += 1;
+}
+
 static bls_status_t enqueue_ring(bls_plan_t *pl, int mode, long long t_last, long long floor_, int k, const int *ids,
                                  const int *off, long long n_ids)
 {
@@ -458,13 +479,15 @@ bls_status_t bls_step(bls_plan_t *pl, int k, const int32_t *ids, const int32_t *
     if (ring) {
         const bls_status_t st = enqueue_ring(pl, BLS_MODE_STEP, t, t - k, k, ids, offsets, n_ids);
         if (st != BLS_OK) return st;
+    } else if (!overlapped && !pl->unserved && small_applies(pl)) {
+        enqueue_small(pl, t, ids, offsets, n_ids);     // posts, answers and completes iteration t on every rank
     } else if (overlapped) {
         enqueue_wave_overlapped(pl, t, t - k, k, ids, offsets, n_ids);
         pl->unserved = 1;                              // iteration t is answered by the next wave
     } else {
         enqueue_wave(pl, BLS_MODE_STEP, t, t - k, k, ids, offsets, n_ids);
     }
-    if (t - k >= 0) {
+    if (t - k >= pl->t_handed) {                       // (an iteration of an earlier loop has been handed back already)
         *out = slot_out(pl, t - k);
         *out_iter = t - k;
         pl->t_handed = t - k + 1;
@@ -661,6 +684,13 @@ bls_status_t bls_set_overlap(bls_plan_t *pl, int mode)
 {
     if (!pl || mode < -1 || mode > 1) return BLS_EINVAL;
     pl->overlap_mode = mode;
+    return BLS_OK;
+}
+
+bls_status_t bls_set_fused(bls_plan_t *pl, int mode)
+{
+    if (!pl || mode < -1 || mode > 1) return BLS_EINVAL;
+    pl->fused_mode = mode;
     return BLS_OK;
 }
 

@@ -108,14 +108,17 @@ __device__ __forceinline__ bool bag_range(const RouteCtx &c, long long g, long l
 // on the table only, so the (requester, table) chunks move as a whole.  Chunk
 // lengths come from the offsets alone; an exclusive scan in (owner, table) order
 // gives every chunk its place in the packed send buffer, and the send counts and
-// displacements follow.
-__device__ __forceinline__ void tw_meta_warp(const BlsParams &p, int src, int lane)
+// displacements follow.  With `publish` the results go to memory (chunk bases, send
+// counts, displacements, end of the last sub-bag); in any case the warp learns where
+// the chunk of pair `want` starts and ends (the fused kernel for small iterations lets
+// every block work that out for itself instead of waiting for another block).
+__device__ __forceinline__ void tw_meta_ctx(const BlsParams &p, const RouteCtx &c, int src, int lane, bool publish,
+                                            int want, int &cb_want, int &cb_after)
 {
-    RouteCtx c;
-    if (!route_ctx(p, src, c)) return;
     const long long g_rank = (long long)src * p.T * p.b;
     int *cb = p.chunk_base + (size_t)src * (p.NI + 1);
     long long run = 0;
+    int mine = 0, after = 0;
     for (int i0 = 0; i0 < p.NI; i0 += 32) {
         const int i = i0 + lane;
         long long n = 0;
@@ -123,18 +126,25 @@ __device__ __forceinline__ void tw_meta_warp(const BlsParams &p, int src, int la
             const long long g0 = g_rank + (long long)p.pair[i].t * p.b;
             const long long a = c.off[g0], e = c.off[g0 + p.b];
             n = e - a;
-            if (a < 0 || n < 0 || e > c.n_ids) { n = 0; flag(p, BLS_ST_EINVAL); }
+            if (a < 0 || n < 0 || e > c.n_ids) { n = 0; if (publish) flag(p, BLS_ST_EINVAL); }
         }
         long long incl = n;
         for (int o = 1; o < 32; o <<= 1) {
             const long long y = __shfl_up_sync(0xffffffffu, incl, o);
             if (lane >= o) incl += y;
         }
-        if (i < p.NI) cb[i] = (int)min(run + incl - n, (long long)0x7fffffff);
+        const int base = (int)min(run + incl - n, (long long)0x7fffffff);
+        if (i < p.NI && publish) cb[i] = base;
+        if (i == want) mine = base;
+        if (i == want + 1) after = base;
         run += __shfl_sync(0xffffffffu, incl, 31);
     }
+    const int total = (int)min(run, (long long)0x7fffffff);
+    cb_want = __shfl_sync(0xffffffffu, mine, want & 31);
+    cb_after = want + 1 < p.NI ? __shfl_sync(0xffffffffu, after, (want + 1) & 31) : total;
+    if (!publish) return;
     if (lane == 0) {
-        cb[p.NI] = (int)min(run, (long long)0x7fffffff);
+        cb[p.NI] = total;
         if (run > p.cap) flag(p, BLS_ST_ENOSPC);
         c.sub_start[p.NQ] = (int)(run > p.cap ? p.cap : run);
     }
@@ -144,6 +154,14 @@ __device__ __forceinline__ void tw_meta_warp(const BlsParams &p, int src, int la
         c.sdispls[d] = lo;
         c.sendcounts[d] = hi - lo;
     }
+}
+
+__device__ __forceinline__ void tw_meta_warp(const BlsParams &p, int src, int lane)
+{
+    RouteCtx c;
+    if (!route_ctx(p, src, c)) return;
+    int first, second;
+    tw_meta_ctx(p, c, src, lane, true, 0, first, second);
 }
 
 // Publish the progress of the wave that has just run (lane r = rank r).  For every

@@ -69,15 +69,17 @@ __device__ __forceinline__ void flush(float *o, const Acc<DT> &acc)
 // One run: nb consecutive sub-bags of pair `pr` requested by rank `src`, starting at
 // sample s0, in ring slot `slot`.  With HOT, lookups whose slot number (written by
 // the router) is below K read their row from the staged copy in shared memory.
+// `end_pos` >= 0 gives the send-buffer position where the run's IDs end, for a caller that
+// knows it while the start of the sub-bag after the run may not be in memory yet.
 template <int LANES, int DT, int U, bool HOT>
 __device__ __forceinline__ void stream_run(const BlsParams &p, const BlsPairDesc &pr, int i, int slot, int src,
-                                           int s0, int nb, int lane, const uint4 *hot_rows)
+                                           int s0, int nb, int lane, const uint4 *hot_rows, int end_pos = -1)
 {
     constexpr int Q = U / 4;                           // 16-byte ID quads per batch
     const size_t bag_stride = (size_t)p.T * p.D;       // floats between consecutive samples in out
     const int *ss = p.sub_start + ((size_t)slot * p.P + src) * (size_t)p.sub_stride + (size_t)i * p.b + s0;
     const int p0 = min(max(ss[0], 0), p.cap);
-    const int n = min(max(ss[nb], p0), p.cap) - p0;    // rows in this run
+    const int n = min(max(end_pos >= 0 ? end_pos : ss[nb], p0), p.cap) - p0;    // rows in this run
     // The ID stream is read in aligned 16-byte quads and processed in whole batches
     // of U rows: stream coordinate y = a + x, where x counts the run's rows and
     // a = p0 mod 4.  The a IDs before the run and the IDs after it up to the end of

@@ -70,7 +70,7 @@ struct BlsDev {
     int onehot[BLS_MAX_SLOTS];                    // table-wise: every bag of the iteration in this slot has exactly one ID
     int work_ctr;                                 // next run of the gather kernel (reset by the gate)
     int done_ctr;                                 // blocks of the wave's last kernel that have finished
-    int pad;
+    int small_ctr;                                // blocks of the fused small-iteration kernel that have finished (its last block resets it)
 };
 
 struct BlsTableDesc {
@@ -174,6 +174,7 @@ struct bls_plan {
     int side_ready;
     int unserved;                 // iterations posted whose answer has not been enqueued yet (0 or 1)
     int overlap_mode;             // -1 never, 0 chosen by the size of an iteration, 1 whenever the mode applies
+    int fused_mode;               // one-launch kernel for small table-wise iterations: -1 never, 0 chosen by size, 1 whenever it applies
 };
 #define BLS_PROF_MAX 1024
 
@@ -189,4 +190,6 @@ void bls_launch_meta(const bls_plan_t *pl, cudaStream_t stream);   // table-wise
 void bls_launch_route(const bls_plan_t *pl);
 void bls_launch_route_beside(const bls_plan_t *pl, cudaStream_t stream);   // table-wise router sized to run beside the gather kernel
 void bls_launch_gather(const bls_plan_t *pl);
+// the whole of iteration t (route, gather, return, ring bookkeeping) in one launch: small table-wise iterations, ranks in lockstep
+void bls_launch_small(const bls_plan_t *pl, long long t, const int *ids, const int *off, long long n_ids);
 int bls_route_kernels(const bls_plan_t *pl);   // kernels bls_launch_route enqueues

@@ -21,24 +21,18 @@ struct TileGiven {
 // First half (chunk lengths, scan, counts, displacements): tw_meta_warp, run by the
 // gate kernel.  Second half, here: move every ID to its place and write the sub-bag
 // starts.
-// grid (NT, P): tile = p.tile_bags bags of one (requester, table) chunk (128 for long
-// bags, up to the whole chunk for short ones, so that a block always has a few
-// thousand IDs to move).  Copies the tile's IDs to their place in the send buffer
-// (coalesced) and writes the sub-bag starts.
-template <int INFLIGHT, class Where>
-__device__ __forceinline__ void tw_copy_tile(const BlsParams &p, const Where where)
+// A tile = p.tile_bags bags of one (requester, table) chunk (128 for long bags, up to the
+// whole chunk for short ones, so that a block always has a few thousand IDs to move); the
+// stand-alone kernel runs on a grid (NT, P).  A block copies the tile's IDs to their place
+// in the send buffer (coalesced) and writes the sub-bag starts.
+// The work on one tile, given the requester's context, the tile (pair i, bags s0 .. s0 + nb - 1 of table t)
+// and the chunk's place (cb) and accepted length (cn) in the send buffer.  Returns the end of the
+// tile's IDs relative to the start of the chunk.
+template <int INFLIGHT>
+__device__ __forceinline__ int tw_copy_ctx(const BlsParams &p, const RouteCtx &c, int src, int i, int t, int s0, int nb,
+                                           int cb, int cn)
 {
-    const int src = where.src();
-    RouteCtx c;
-    if (!route_ctx(p, src, c)) return;
-    const int i = where.tile() / p.tiles_per_table;
-    const int s0 = (where.tile() % p.tiles_per_table) * p.tile_bags;
-    const int nb = min(p.tile_bags, p.b - s0);
-    const int t = p.pair[i].t;
     const long long g0 = ((long long)src * p.T + t) * p.b;
-    const int *cbp = p.chunk_base + (size_t)src * (p.NI + 1);
-    const int cb = cbp[i];
-    const int cn = cbp[i + 1] - cb;              // chunk length accepted by the meta kernel
     const long long off0 = c.off[g0];
     __shared__ int s_lo, s_hi;
     bool other_length = false;                   // a bag that does not hold exactly one ID
@@ -87,6 +81,20 @@ __device__ __forceinline__ void tw_copy_tile(const BlsParams &p, const Where whe
             if (pos < p.cap) { c.sendbuf[pos] = id; hs[pos] = (unsigned short)slot; }
         }
     }
+    return hi;
+}
+
+template <int INFLIGHT, class Where>
+__device__ __forceinline__ void tw_copy_tile(const BlsParams &p, const Where where)
+{
+    const int src = where.src();
+    RouteCtx c;
+    if (!route_ctx(p, src, c)) return;
+    const int i = where.tile() / p.tiles_per_table;
+    const int s0 = (where.tile() % p.tiles_per_table) * p.tile_bags;
+    const int *cbp = p.chunk_base + (size_t)src * (p.NI + 1);
+    const int cb = cbp[i];
+    tw_copy_ctx<INFLIGHT>(p, c, src, i, p.pair[i].t, s0, min(p.tile_bags, p.b - s0), cb, cbp[i + 1] - cb);
 }
 
 

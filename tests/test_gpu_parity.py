@@ -38,7 +38,8 @@ def make_plan(w, tabs, k_max, cap=None):
     plan = bls.bls_plan(tabs, w.partition, w.P, w.local_batch, k_max, cap)
     bls.bls_set_poison(plan, True)          # every bag must be written: an unwritten one would show up as NaN
     bls.bls_set_overlap(plan, 1)            # test workloads are small: use the overlapped mode wherever it applies
-    return plan
+    bls.bls_set_fused(plan, -1)             # ... and the stand-alone kernels, not the one-launch kernel for small iterations,
+    return plan                             # which has tests of its own (test_gpu_fused.py)
 
 
 def check_route(w, view, ids, off, recv_side=True):

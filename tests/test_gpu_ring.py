@@ -22,13 +22,17 @@ def assert_matches_oracle(w, data, inputs, outs):
         assert err <= TOL[w.tables[0].dtype], (it, err)
 
 
-def run_loop(w, tabs, k, n_iter, k_max=None, stalls=None, check_views=False, wait_limit=None, ring=None):
+def run_loop(w, tabs, k, n_iter, k_max=None, stalls=None, check_views=False, wait_limit=None, ring=None, fused=False):
     """Listing 2's loop: n_iter steps then the drain; returns {iteration: output}.
     ring = 1 runs every call as one launch of the persistent ring kernel (which is also what
-    injected delays switch on); None leaves the plan's default (stand-alone kernels)."""
+    injected delays switch on); None leaves the plan's default (stand-alone kernels).
+    fused: every step of a table-wise plan is one launch of the kernel for small iterations."""
     plan = make_plan(w, tabs, k if k_max is None else k_max)
     if ring is not None:
         bls.bls_set_ring(plan, ring)
+    if fused:
+        bls.bls_set_overlap(plan, -1)
+        bls.bls_set_fused(plan, 1)
     if wait_limit is not None:
         bls.bls_set_wait_limit(plan, wait_limit)
     for r, ns in (stalls or {}).items():
@@ -62,22 +66,26 @@ def run_loop(w, tabs, k, n_iter, k_max=None, stalls=None, check_views=False, wai
     return outs, inputs, status, lag
 
 
-@pytest.mark.parametrize("ring", [None, 1], ids=["kernels", "ring"])
+@pytest.mark.parametrize("ring", [None, 1, "fused"], ids=["kernels", "ring", "fused"])
 @pytest.mark.parametrize("num,rs,bs", [(1, 1.0, 1.0), (3, 0.01, 0.02), (4, 0.002, 0.01), (5, 0.001, 0.003)])
 def test_output_is_independent_of_k(num, rs, bs, ring):
     w = bi.workload(num, rs, bs)
+    fused = ring == "fused"
+    if fused and w.partition != "table_rr":
+        pytest.skip("the one-launch kernel exists for table-wise placement")
+    ring = None if fused else ring
     data = [bi.table_values(t) for t in w.tables]
     tabs = dev_tables(w, data)
     n_iter = 7
-    ref, inputs, status, lag = run_loop(w, tabs, 0, n_iter, check_views=True, ring=ring)
+    ref, inputs, status, lag = run_loop(w, tabs, 0, n_iter, check_views=True, ring=ring, fused=fused)
     assert status == bls.BLS_OK and lag == 0 and sorted(ref) == list(range(n_iter))
     P, T, b = w.P, w.T, w.local_batch
     for it, (ids, off) in enumerate(inputs):
         want = oracle.pool_definition(P, T, b, w.tables, data, ids, off)
         assert oracle.vector_rel_err(ref[it].cpu().numpy(), want) <= TOL[w.tables[0].dtype]
     for k in (1, 2, 4, 8):
-        outs, _, status, lag = run_loop(w, tabs, k, n_iter, check_views=True, ring=ring)
-        assert status == bls.BLS_OK and lag <= k
+        outs, _, status, lag = run_loop(w, tabs, k, n_iter, check_views=True, ring=ring, fused=fused)
+        assert status == bls.BLS_OK and lag <= (0 if fused else k)
         assert sorted(outs) == list(range(n_iter))
         for it in range(n_iter):
             assert torch.equal(outs[it], ref[it]), (k, it)           # deterministic kernels: bit-identical
