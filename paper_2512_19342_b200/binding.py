@@ -346,30 +346,37 @@ class A2a:
         self.handle = C.c_void_p()
         _check(lib().bls_a2a_create(P, k_max, C.c_int64(max_bytes_per_rank), C.c_void_p(self.workspace.data_ptr()),
                                     C.c_size_t(n.value), _stream_ptr(stream), C.byref(self.handle)), "bls_a2a_create")
-        self._keep = []
+        self._borrowed = collections.deque(maxlen=k_max + 2)   # buffers of the requests still in flight
+        self._views = {}                     # receive slot address -> the three tensor views of that slot
+        self._ret = (C.c_void_p(), C.c_int64(0), C.c_void_p(), C.c_void_p(), C.c_int64(-1))
+        self._ret_refs = tuple(C.byref(x) for x in self._ret)
+        l = lib()
+        l.bls_a2a_post.argtypes = [C.c_void_p, C.c_void_p, C.c_int64, C.c_void_p, C.c_void_p, C.c_int64]
+        l.bls_a2a_wait.argtypes = [C.c_void_p] * 6
 
     def post(self, sendbuf: torch.Tensor, sendcounts: torch.Tensor, sdispls: torch.Tensor, max_segment_bytes: int):
         """sendbuf uint8 [P][stride]; sendcounts/sdispls int64 [P][P] (bytes), all on the device."""
-        self._keep.append((sendbuf, sendcounts, sdispls))
-        del self._keep[:-(self.k_max + 2)]
-        _check(lib().bls_a2a_post(self.handle, C.c_void_p(sendbuf.data_ptr()), C.c_int64(sendbuf.shape[1]),
-                                  C.c_void_p(sendcounts.data_ptr()), C.c_void_p(sdispls.data_ptr()),
-                                  C.c_int64(max_segment_bytes)), "bls_a2a_post")
+        self._borrowed.append((sendbuf, sendcounts, sdispls))
+        _check(lib().bls_a2a_post(self.handle, sendbuf.data_ptr(), sendbuf.shape[1], sendcounts.data_ptr(),
+                                  sdispls.data_ptr(), max_segment_bytes), "bls_a2a_post")
 
     def wait(self):
         """Completes the oldest request: (recv uint8 [P][stride], recvcounts, rdispls int64 [P][P], request number)."""
-        recv, rc, rd = C.c_void_p(), C.c_void_p(), C.c_void_p()
-        stride, req = C.c_int64(0), C.c_int64(-1)
-        _check(lib().bls_a2a_wait(self.handle, C.byref(recv), C.byref(stride), C.byref(rc), C.byref(rd), C.byref(req)),
-               "bls_a2a_wait")
-        ws, P = self.workspace, self.P
+        recv, stride, rc, rd, req = self._ret
+        _check(lib().bls_a2a_wait(self.handle, *self._ret_refs), "bls_a2a_wait")
+        key = (recv.value, stride.value)
+        views = self._views.get(key)
+        if views is None:
+            ws, P = self.workspace, self.P
 
-        def view(ptr, nbytes):
-            off = ptr - ws.data_ptr()
-            return ws[off:off + nbytes]
-        return (view(recv.value, P * stride.value).view(P, stride.value),
-                view(rc.value, 8 * P * P).view(torch.int64).view(P, P),
-                view(rd.value, 8 * P * P).view(torch.int64).view(P, P), req.value)
+            def view(ptr, nbytes):
+                off = ptr - ws.data_ptr()
+                return ws[off:off + nbytes]
+            views = (view(recv.value, P * stride.value).view(P, stride.value),
+                     view(rc.value, 8 * P * P).view(torch.int64).view(P, P),
+                     view(rd.value, 8 * P * P).view(torch.int64).view(P, P))
+            self._views[key] = views
+        return views + (req.value,)
 
     def status(self) -> int:
         return lib().bls_a2a_status(self.handle)

@@ -13,7 +13,7 @@
 // dst lands at rdispls[dst][src] = sum of the counts of lower-ranked sources, which
 // every block derives from the count matrix itself.
 #include <stdlib.h>
-#include "bls_internal.h"
+#include "bls_device.cuh"
 
 struct bls_a2a {
     int P, S;
@@ -85,6 +85,7 @@ __device__ __forceinline__ bool a2a_accept(const A2aArgs &a, int src, int dst, l
 // with stride gridDim.x, so a segment of any length is covered whatever the host's size hint was.
 __global__ void __launch_bounds__(256) bls_a2a_put_kernel(A2aArgs a, long long chunk_bytes)
 {
+    stream_order_enter();
     const int src = blockIdx.y / a.P, dst = blockIdx.y % a.P;
     long long n, rd;
     int why;
@@ -146,6 +147,7 @@ __global__ void __launch_bounds__(256) bls_a2a_put_kernel(A2aArgs a, long long c
 // slot was completed before its request had run).
 __global__ void bls_a2a_complete_kernel(int *arrived, int P, int *status)
 {
+    stream_order_enter();
     const int r = threadIdx.x;
     if (r < P) {
         if (arrived[r] != P) atomicOr(status, BLS_ST_ESTATE);
@@ -221,7 +223,8 @@ bls_status_t bls_a2a_post(bls_a2a_t *h, const void *sendbuf, int64_t send_stride
     chunk_bytes = (chunk_bytes + 15) / 16 * 16;
     chunks = max_segment_bytes > 0 ? (max_segment_bytes + chunk_bytes - 1) / chunk_bytes : 1;
     if (chunks > 65535) return BLS_EINVAL;
-    bls_a2a_put_kernel<<<dim3((unsigned)chunks, h->P * h->P), 256, 0, h->stream>>>(a, chunk_bytes);
+    // (small messages are bound by the latency between dependent launches: see stream_order_enter)
+    launch_serialised(bls_a2a_put_kernel, dim3((unsigned)chunks, h->P * h->P), dim3(256), h->stream, a, chunk_bytes);
     h->posted++;
     return cudaGetLastError() == cudaSuccess ? BLS_OK : BLS_ECUDA;
 }
@@ -232,7 +235,7 @@ bls_status_t bls_a2a_wait(bls_a2a_t *h, const void **recv, int64_t *recv_stride,
     if (!h) return BLS_EINVAL;
     if (h->completed == h->posted) return BLS_ESTATE;                 // nothing outstanding
     const int slot = (int)(h->completed % h->S);
-    bls_a2a_complete_kernel<<<1, 32, 0, h->stream>>>(h->arrived + (size_t)slot * h->P, h->P, h->status);
+    launch_serialised(bls_a2a_complete_kernel, dim3(1), dim3(32), h->stream, h->arrived + (size_t)slot * h->P, h->P, h->status);
     if (recv) *recv = h->recv + (size_t)slot * h->P * h->cap;
     if (recv_stride) *recv_stride = h->cap;
     if (recvcounts) *recvcounts = (const int64_t *)(h->recvcounts + (size_t)slot * h->P * h->P);

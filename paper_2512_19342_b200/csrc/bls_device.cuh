@@ -10,6 +10,35 @@ __device__ __forceinline__ unsigned long long globaltimer_ns()
     return t;
 }
 
+// Programmatic stream serialisation, for chains of very short kernels.  A kernel launched with
+// launch_serialised() may have its blocks made resident while the previous kernel of the stream is
+// still running; stream_order_enter(), the first statement of every such kernel, holds them until
+// that kernel has completed and its writes are visible, and then lets the next kernel of the stream
+// be brought in the same way.  The order of the stream is unchanged; the launch latency between
+// dependent kernels is hidden.  Because every kernel launched this way waits before anything
+// else, completion stays transitive along the stream.
+__device__ __forceinline__ void stream_order_enter()
+{
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+}
+
+template <class... Params, class... Args>
+static inline cudaError_t launch_serialised(void (*kernel)(Params...), dim3 grid, dim3 block, cudaStream_t stream,
+                                            Args... args)
+{
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, Params(args)...);
+}
+
 __device__ __forceinline__ void flag(const BlsParams &p, int bit) { atomicOr(&p.dev->status, bit); }
 
 // Injected delay of rank r before it posts iteration j: the fixed part plus a uniform draw

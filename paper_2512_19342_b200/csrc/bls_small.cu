@@ -24,12 +24,7 @@ bls_small_tw_kernel(BlsParams p, long long t, const int *ids, const int *off, lo
 {
     __shared__ int s_meta[3];                          // ranks in lockstep?  start and end of the block's chunk
     __shared__ int s_last;
-    // Launched with programmatic stream serialisation: the blocks may become resident while the
-    // previous kernel of the stream is still running, and wait here until it has completed and its
-    // writes are visible - the order of the stream is kept, the launch latency is hidden.  The next
-    // kernel of the stream may then be brought in the same way.
-    asm volatile("griddepcontrol.wait;" ::: "memory");
-    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    stream_order_enter();                              // launched with launch_serialised()
     BlsDev *d = p.dev;
     const int src = blockIdx.y;
     const int i = blockIdx.x / p.tiles_per_table;      // (owner, table) pair of the tile
@@ -107,16 +102,8 @@ bls_small_tw_kernel(BlsParams p, long long t, const int *ids, const int *off, lo
 template <int LANES, int DT>
 static void launch_small_kernel(const bls_plan_t *pl, long long t, const int *ids, const int *off, long long n_ids)
 {
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(pl->prm.NT, pl->prm.P);
-    cfg.blockDim = dim3(BLS_ROUTE_TB);
-    cfg.stream = pl->stream;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = 1;
-    cfg.attrs = attr;
-    cfg.numAttrs = 1;
-    cudaLaunchKernelEx(&cfg, bls_small_tw_kernel<LANES, DT>, pl->prm, t, ids, off, n_ids);
+    launch_serialised(bls_small_tw_kernel<LANES, DT>, dim3(pl->prm.NT, pl->prm.P), dim3(BLS_ROUTE_TB), pl->stream,
+                      pl->prm, t, ids, off, n_ids);
 }
 
 template <int DT>
