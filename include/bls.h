@@ -160,7 +160,9 @@ bls_status_t bls_drain(bls_plan_t *plan, const float **out /*host out*/, int64_t
  * to a staging area of the ring (pinned memory recommended), and the iteration
  * handed back, if any, is copied to host_out (fp32 [P][b][T][dim]; may be NULL to
  * skip the copy).  The copies run asynchronously on two internal streams (upload of the
- * next iteration and download of the previous result overlap); the plan's stream waits for
+ * next iteration and download of the previous result overlap; with a bound k >= 1 - k >= 2 in
+ * overlapped mode - and no injected delays the download of iteration t-k also runs beside the
+ * kernels of iteration t, which work on other slots of the ring); the plan's stream waits for
  * them, so synchronising it, or enqueuing work on it, after the call sees host_out complete.
  * The host buffers must stay untouched until then. */
 bls_status_t bls_step_host(bls_plan_t *plan, int k, const int32_t *ids /*host*/,

@@ -528,8 +528,8 @@ bls_status_t bls_drain(bls_plan_t *pl, const float **out, int64_t *out_iter)
 }
 
 // Host-buffer path: the copies run on two streams of their own so that the upload of the
-// next iteration and the download of the previous result overlap (PCIe is full duplex) and
-// only the kernels sit between them.  The plan's stream waits for both, so work enqueued
+// next iteration and the download of the previous result overlap (PCIe is full duplex); with a
+// bound >= 1 the download of iteration t - k also runs beside the kernels of iteration t.  The plan's stream waits for both, so work enqueued
 // on it afterwards, and a synchronisation of it, see the copies complete.
 static bool host_path_ready(bls_plan_t *pl)
 {
@@ -542,21 +542,30 @@ static bool host_path_ready(bls_plan_t *pl)
         return false;
     // nothing has been enqueued on the copy streams yet: order them after what the plan's stream holds
     if (cudaEventRecord(pl->e_comp, pl->stream) != cudaSuccess) return false;
+    pl->comp_iter = pl->t_next;
     pl->host_path = 1;
     return true;
 }
 
-static bls_status_t download(bls_plan_t *pl, const float *out, float *host_out)
+// Copy a handed-back iteration to the host.  `early`: the iteration was complete before the kernels
+// that the current call has just enqueued (a bound >= 1; >= 2 in overlapped mode, where an iteration
+// is answered one step after it was posted), and those kernels write another slot of the ring, so
+// the copy only has to wait for the previous call's kernels and runs beside the current ones.
+static bls_status_t download(bls_plan_t *pl, const float *out, float *host_out, bool early)
 {
-    if (cudaEventRecord(pl->e_comp, pl->stream) != cudaSuccess) return BLS_ECUDA;
-    if (out && host_out) {
+    const bool copy = out && host_out;
+    if (!early && cudaEventRecord(pl->e_comp, pl->stream) != cudaSuccess) return BLS_ECUDA;
+    if (copy) {
+        // (early: e_comp still marks the end of the previous call's kernels)
         if (cudaStreamWaitEvent(pl->s_out, pl->e_comp, 0) != cudaSuccess ||
             cudaMemcpyAsync(host_out, out, sizeof(float) * (size_t)pl->prm.out_slot_elems, cudaMemcpyDeviceToHost,
                             pl->s_out) != cudaSuccess ||
-            cudaEventRecord(pl->e_out, pl->s_out) != cudaSuccess ||
-            cudaStreamWaitEvent(pl->stream, pl->e_out, 0) != cudaSuccess)
+            cudaEventRecord(pl->e_out, pl->s_out) != cudaSuccess)
             return BLS_ECUDA;
     }
+    if (early && cudaEventRecord(pl->e_comp, pl->stream) != cudaSuccess) return BLS_ECUDA;
+    pl->comp_iter = pl->t_next;
+    if (copy && cudaStreamWaitEvent(pl->stream, pl->e_out, 0) != cudaSuccess) return BLS_ECUDA;
     return BLS_OK;
 }
 
@@ -580,10 +589,14 @@ bls_status_t bls_step_host(bls_plan_t *pl, int k, const int32_t *ids, const int3
         cudaEventRecord(pl->e_in, pl->s_in) != cudaSuccess ||
         cudaStreamWaitEvent(pl->stream, pl->e_in, 0) != cudaSuccess)
         return BLS_ECUDA;
+    // e_comp marks the end of the previous iteration's kernels only if that iteration came through this path too
+    const bool fresh = pl->comp_iter == pl->t_next;
     const float *out = nullptr;
     bls_status_t st = bls_step(pl, k, d_ids, d_off, n_ids, &out, out_iter);
     if (st != BLS_OK) return st;
-    return download(pl, out, host_out);
+    // with injected delays (ring kernel) an iteration may complete inside the launch that hands it back
+    const bool early = out && fresh && !ring_applies(pl) && !pl->ring_used && k >= (pl->unserved ? 2 : 1);
+    return download(pl, out, host_out, early);
 }
 
 bls_status_t bls_drain_host(bls_plan_t *pl, float *host_out, int64_t *out_iter)
@@ -593,7 +606,7 @@ bls_status_t bls_drain_host(bls_plan_t *pl, float *host_out, int64_t *out_iter)
     const float *out = nullptr;
     bls_status_t st = bls_drain(pl, &out, out_iter);
     if (st != BLS_OK) return st;
-    return download(pl, out, host_out);
+    return download(pl, out, host_out, false);
 }
 
 bls_status_t bls_view(bls_plan_t *pl, int64_t iter, bls_route_view_t *v)

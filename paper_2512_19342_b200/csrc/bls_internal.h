@@ -155,6 +155,7 @@ struct bls_plan {
     cudaStream_t s_in, s_out;
     cudaEvent_t e_in, e_comp, e_out;
     int host_path;
+    long long comp_iter;          // value of t_next when e_comp was last recorded (it then marks the end of iteration t_next - 1)
     long long kernels_launched;   // total kernels enqueued through this plan
     int any_stall;                // a delay was injected at some point: ranks may be out of lockstep
     int bags_per_run;             // gather kernel: consecutive sub-bags streamed by one lane group

@@ -257,6 +257,40 @@ def test_host_buffer_entry_points():
         assert oracle.vector_rel_err(got[it].numpy(), want) <= 1e-5
 
 
+@pytest.mark.parametrize("mode,k,k_max", [("overlapped", 1, 1), ("overlapped", 2, 2), ("overlapped", 4, 4), ("overlapped", 2, 5),
+                                          ("kernels", 0, 0), ("kernels", 1, 1), ("kernels", 3, 3), ("fused", 1, 1), ("fused", 2, 4)])
+def test_host_buffer_loop_without_synchronisation(mode, k, k_max):
+    """The host-buffer calls back to back, nothing synchronised until the end: uploads, kernels and
+    downloads of different iterations overlap (with a bound >= 1 the download of iteration t - k runs
+    beside the kernels of iteration t).  Every slot is filled with NaN patterns before it is reused,
+    so a download that read its slot too late, or a kernel that wrote it too early, would show."""
+    w = bi.workload(3, 0.02, 0.05)
+    data = [bi.table_values(t) for t in w.tables]
+    tabs = dev_tables(w, data)
+    plan = make_plan(w, tabs, k_max)                    # poison on, overlapped mode wherever it applies, one-launch kernel off
+    if mode != "overlapped":
+        bls.bls_set_overlap(plan, -1)
+    if mode == "fused":
+        bls.bls_set_fused(plan, 1)
+    n = 9
+    inputs = [bi.make_iteration(w, t) for t in range(n)]
+    pinned = [(torch.from_numpy(i).pin_memory(), torch.from_numpy(o).pin_memory()) for i, o in inputs]
+    host_out = [torch.full((w.P, w.local_batch, w.T, w.tables[0].dim), float("nan")).pin_memory() for _ in range(n)]
+    handed = []
+    for t in range(n):
+        it = bls.bls_step_host(plan, k, *pinned[t], host_out[len(handed)])
+        if it >= 0:
+            handed.append(it)
+    while True:
+        it = bls.bls_drain_host(plan, host_out[len(handed)] if len(handed) < n else None)
+        if it < 0:
+            break
+        handed.append(it)
+    torch.cuda.synchronize()
+    assert handed == list(range(n)) and bls.bls_status(plan)[0] == bls.BLS_OK
+    assert_matches_oracle(w, data, inputs, dict(enumerate(host_out)))
+
+
 def host_delays(P, n_iter, fixed_ns, span_ns, seed):
     """The delays the device draws, reproduced on the host: delay of rank r before iteration j =
     fixed + (SplitMix64 output for state seed + ((r << 40) + j + 1) * golden ratio) mod (span + 1)."""
