@@ -140,7 +140,7 @@ bls_status_t bls_lookup(bls_plan_t *plan, int64_t iter);
  *           a million lookups or more (bls_set_overlap), a step works in overlapped mode (the
  *           paper's Table I: communication of one batch beside computation of another):
  *           the requesters post iteration t while the owners answer iteration t-1, the
- *           router running on a second stream beside the gather-pool kernel.  The
+ *           router enqueued on a second stream beside the gather-pool kernel.  The
  *           plan's stream waits for that second stream before the call returns control of
  *           it, so the caller sees one ordered stream.  In this mode the owners are one
  *           iteration behind the requesters after a step (bls_status reports a lag of 1)

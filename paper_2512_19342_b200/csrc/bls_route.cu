@@ -14,9 +14,10 @@
 // Row-wise placement: a real multisplit, done per tile of 128 bags of one table.
 #include "bls_route.cuh"
 
-// Blocks of 128 threads and at most 32 registers: one such block fits on every SM beside
-// the resident blocks of the gather kernel (3 x 256 threads x 80 registers), so that the
-// router can work on the next iteration while the previous one is answered.
+// Blocks of 128 threads and at most 32 registers, 16 to an SM.  In overlapped mode the kernel sits on
+// a second stream behind the gather kernel (3 x 256 threads x 80 registers per SM); measured, its
+// blocks come in as the gather kernel's retire (kernels whose L1 / shared-memory splits differ are
+// not made resident together) and the small blocks fill that tail quickly.
 __global__ void __launch_bounds__(128, 16) bls_tw_copy_kernel(BlsParams p) { tw_copy_tile<8>(p, TileFromGrid()); }
 
 __global__ void __launch_bounds__(BLS_ROUTE_TB, 8) bls_rw_count_kernel(BlsParams p) { rw_count_tile(p, TileFromGrid()); }
