@@ -330,9 +330,9 @@ static void enqueue_wave(bls_plan_t *pl, int mode, long long t_last, long long f
 // iteration t - 1, which is in another slot, so the two do not depend on each other
 // (Table I of the paper: communication of one batch beside computation of another).  The
 // gate plans both; then the gather kernel (answer t - 1, commit) goes to the plan's stream
-// and the router's two kernels (post t) to a second stream: gate, launch gaps and the router's
-// first half leave the critical path, and the copy kernel's small blocks fill the gather kernel's
-// tail as its blocks retire (measured: they are not resident together before that, and making
+// and the router's two kernels (post t) to a second stream: the router's first half and the launch
+// gap between router and gather kernel leave the critical path, and the copy kernel's small blocks
+// fill the gather kernel's tail as its blocks retire (measured: they are not resident together before that, and making
 // them so by equal L1 / shared-memory splits gains nothing).  (Row-wise placement stays sequential:
 // its router needs shared memory and several blocks per SM to hide its load latency,
 // neither of which the resident gather blocks leave.)  The plan's stream waits for the copy
