@@ -9,7 +9,7 @@ from __future__ import annotations
 import collections
 import ctypes as C
 import os
-from typing import List, Optional, Sequence, Tuple
+from typing import Optional, Sequence
 
 import torch
 
