@@ -146,7 +146,8 @@ bls_status_t bls_lookup(bls_plan_t *plan, int64_t iter);
  *           iteration behind the requesters after a step (bls_status reports a lag of 1)
  *           and the first bls_drain call enqueues the last answer.  Results are the same
  *           bit for bit in both modes.
- *           Small table-wise iterations without injected delays (below about 256 K lookups;
+ *           Small table-wise iterations without injected delays (below about 256 K lookups,
+ *           below a million when bags hold four IDs or fewer on average;
  *           bls_set_fused) are ONE kernel launch: every block routes a tile of one
  *           (requester, table) chunk and answers it at once, the last block publishes the
  *           iteration for all ranks.  Same routing artefacts, same sums, bit for bit.
@@ -220,7 +221,8 @@ bls_status_t bls_timeline(bls_plan_t *plan, int64_t first_iter, int n_iter, uint
 bls_status_t bls_set_overlap(bls_plan_t *plan, int mode);
 /* One-launch iterations (see bls_step): mode 0 (default) uses the fused kernel when an iteration
  * holds fewer than about 256 K lookups (P * max_ids_per_rank < 2^18: below that the launches of a
- * wave cost more than the work in them), 1 whenever it applies (table-wise placement, no injected
+ * wave cost more than the work in them; < 2^20 when max_ids_per_rank allows at most four IDs per bag on
+ * average, where routing and answering a tile in one go stays ahead for longer), 1 whenever it applies (table-wise placement, no injected
  * delays, ring kernel and overlapped mode not in use, no hot-row staging, default tuning), -1 never.
  * May be called at any time. */
 bls_status_t bls_set_fused(bls_plan_t *plan, int mode);

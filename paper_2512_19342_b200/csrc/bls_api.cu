@@ -320,7 +320,6 @@ static void enqueue_wave(bls_plan_t *pl, int mode, long long t_last, long long f
     bls_launch_gate(pl, mode, t_last, floor_, k, ids, off, n_ids);
     bls_launch_route(pl);
     if (ev) cudaEventRecord(ev[1], pl->stream);
-    pl->serve_n_ids = pl->n_ids_of[t_last % pl->prm.S];   // without delays a wave answers the newest iteration
     bls_launch_gather(pl);                             // its last block commits the wave
     if (ev) { cudaEventRecord(ev[2], pl->stream); cudaEventRecord(ev[3], pl->stream); }
     pl->kernels_launched += 2 + bls_route_kernels(pl);
@@ -359,7 +358,6 @@ static void enqueue_wave_overlapped(bls_plan_t *pl, long long t_last, long long 
     bls_launch_gate(pl, BLS_MODE_STEP, t_last, floor_, k, ids, off, n_ids, 1);
     cudaEventRecord(pl->e_fork, pl->stream);
     if (ev) cudaEventRecord(ev[1], pl->stream);
-    pl->serve_n_ids = t_last >= 1 ? pl->n_ids_of[(t_last - 1) % pl->prm.S] : -1;   // the owners answer iteration t - 1
     bls_launch_gather(pl);                             // first, so that its blocks are resident first
     cudaStreamWaitEvent(pl->s_side, pl->e_fork, 0);
     bls_launch_meta(pl, pl->s_side);                   // chunk bases, send counts and displacements of iteration t
@@ -383,15 +381,20 @@ static bool ring_applies(const bls_plan_t *pl)
            (long long)pl->prm.P * pl->prm.cap < (1 << 17);
 }
 
-// Small table-wise iterations with the ranks in lockstep: the whole iteration in one launch
-// (bls_small.cu).  Measured against the wave of stand-alone kernels it is 2.5 times faster at
-// 50 K lookups per iteration, 1.7 times at 200 K, and level from about 350 K (20-ID bags) to
-// 1 M (one-ID bags) lookups.
+// Table-wise iterations with the ranks in lockstep, the whole iteration in one launch (bls_small.cu).
+// Measured against the wave of stand-alone kernels: 2.5 times faster at 50 K lookups per iteration
+// and 1.7 times at 200 K whatever the bag lengths; level from about 350 K lookups with 20-ID bags;
+// with short bags (one ID per bag, or the 2.4 of a Pareto law; 64- and 256-byte rows) still 10-30 %
+// faster at 0.5-1 M lookups, level at 2 M, slower beyond.  At a million lookups the overlapped mode
+// takes over for bounds >= 1 anyway.
 static bool small_applies(const bls_plan_t *pl)
 {
     const BlsParams &p = pl->prm;
     if (pl->fused_mode < 0 || p.part != BLS_PART_TABLE_RR || p.hot.enabled || pl->rows_in_flight != 4) return false;
-    return pl->fused_mode > 0 || (long long)p.P * p.cap < (1 << 18);
+    if (pl->fused_mode > 0) return true;
+    const long long room = (long long)p.P * p.cap;     // lookups an iteration can hold
+    const bool short_bags = (long long)p.cap <= 4LL * p.T * p.b;
+    return room < (1 << 18) || (short_bags && room < (1 << 20));
 }
 
 static void enqueue_small(bls_plan_t *pl, long long t, const int *ids, const int *off, long long n_ids)
@@ -439,7 +442,6 @@ bls_status_t bls_route(bls_plan_t *pl, int64_t iter, const int32_t *ids, const i
     if (!pl || !offsets || (!ids && n_ids > 0) || n_ids < 0) return BLS_EINVAL;
     if (iter != pl->t_next || pl->t_handed != pl->t_next || pl->routed_only >= 0) return BLS_ESTATE;
     poison_slot(pl, iter);
-    pl->n_ids_of[iter % pl->prm.S] = n_ids;
     bls_launch_gate(pl, BLS_MODE_ROUTE_ONLY, iter, -1, 0, ids, offsets, n_ids);
     bls_launch_route(pl);
     bls_launch_commit(pl);
@@ -454,7 +456,6 @@ bls_status_t bls_lookup(bls_plan_t *pl, int64_t iter)
     if (!pl) return BLS_EINVAL;
     if (pl->routed_only != iter) return BLS_ESTATE;
     bls_launch_gate(pl, BLS_MODE_LOOKUP_ONLY, iter, -1, 0, nullptr, nullptr, 0);
-    pl->serve_n_ids = pl->n_ids_of[iter % pl->prm.S];
     bls_launch_gather(pl);                             // its last block commits the wave
     pl->kernels_launched += 2;
     pl->routed_only = -1;
@@ -471,7 +472,6 @@ bls_status_t bls_step(bls_plan_t *pl, int k, const int32_t *ids, const int32_t *
     pl->k_cur = k;
     const long long t = pl->t_next++;
     poison_slot(pl, t);
-    pl->n_ids_of[t % pl->prm.S] = n_ids;
     // (iterations below about a million lookups are bound by the launch rate, of the host or of
     // the GPU, and the second stream costs five more driver calls per step: they stay on one stream)
     const bool ring = ring_applies(pl);

@@ -223,7 +223,6 @@ __device__ __forceinline__ void ring_scheduler(const BlsParams &p, const RingArg
         d->in_ids[slot] = a.ids;
         d->in_off[slot] = a.off;
         d->in_n[slot] = a.n_ids;
-        d->onehot[slot] = 0;                            // the short cut for one-ID bags belongs to the stand-alone gather kernel
     }
     long long posted = act ? d->posted[r] : BIG;
     long long served = act ? d->served[r] : BIG;

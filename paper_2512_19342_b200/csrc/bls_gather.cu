@@ -54,65 +54,6 @@ bls_gather_pool_kernel(BlsParams p, int R, int runs_per_chunk, int n_runs)
     finish_wave(p);
 }
 
-// One-hot iterations (one ID in every bag: the shape of the click-log datasets, Section V-F).  The host
-// launches this kernel instead of the one above when the iteration has exactly one ID per bag on
-// average; the router has recorded whether every bag really holds one (BlsDev::onehot).  If so: no
-// streaming, no run hand-out - a lane group takes bags (pair, requester, sample) in a fixed stride,
-// reads the sub-bag's position, its ID and its row, and stores 0 + row (the same arithmetic as the
-// streaming path, so the bits agree), four bags in flight per lane group.  If not, the kernel does
-// what the streaming kernel does.
-template <int LANES, int DT>
-__global__ void __launch_bounds__(256, 3)
-bls_gather_onehot_kernel(BlsParams p, int R, int runs_per_chunk, int n_runs)
-{
-    BlsDev *dev = p.dev;
-    const long long j0 = dev->serve_iter[p.pair[0].dst];
-    if (j0 < 0 || !dev->onehot[(int)(j0 % p.S)]) {
-        pool_runs<LANES, DT, 4>(p, R, runs_per_chunk, n_runs);
-        finish_wave(p);
-        return;
-    }
-    const int lane = threadIdx.x % LANES;
-    const int slot = (int)(j0 % p.S);
-    const long long nbags = (long long)p.NI * p.P * p.b;
-    const long long stride = (long long)gridDim.x * (blockDim.x / LANES);
-    for (long long g0 = (long long)blockIdx.x * (blockDim.x / LANES) + threadIdx.x / LANES; g0 < nbags; g0 += 4 * stride) {
-        int id[4];
-        const uint4 *row[4];
-        float *o[4];
-        #pragma unroll
-        for (int u = 0; u < 4; u++) {
-            const long long gb = g0 + u * stride;
-            id[u] = -1;
-            if (gb < nbags) {
-                const int i = (int)(gb / ((long long)p.P * p.b));
-                const int rem = (int)(gb - (long long)i * p.P * p.b);
-                const int src = rem / p.b, s = rem - src * p.b;
-                const BlsPairDesc pr = p.pair[i];
-                if (dev->serve_iter[pr.dst] == j0) {
-                    const int pos = p.sub_start[((size_t)slot * p.P + src) * (size_t)p.sub_stride + (size_t)i * p.b + s];
-                    id[u] = __ldcs(p.sendbuf + ((size_t)slot * p.P + src) * (size_t)p.cap + min(max(pos, 0), p.cap - 1)) & 0x7fffffff;
-                    row[u] = reinterpret_cast<const uint4 *>(pr.base) + (size_t)min((unsigned)id[u], (unsigned)pr.nrows - 1u) * LANES + lane;
-                    o[u] = p.out + (size_t)slot * p.out_slot_elems + (((size_t)src * p.b + s) * p.T + pr.t) * p.D + lane * Acc<DT>::N;
-                }
-            }
-        }
-        uint4 v[4];
-        #pragma unroll
-        for (int u = 0; u < 4; u++)
-            if (id[u] >= 0) v[u] = __ldg(row[u]);
-        #pragma unroll
-        for (int u = 0; u < 4; u++)
-            if (id[u] >= 0) {
-                Acc<DT> acc;
-                acc.zero();
-                acc.add(v[u]);
-                flush<DT>(o[u], acc);
-            }
-    }
-    finish_wave(p);
-}
-
 // Bulk-copy variant of the table-wise gather kernel (optional, bls_set_tuning): rows are staged
 // in shared memory by cp.async.bulk, NST stages of BR rows per lane group.  Blocks of 128
 // threads; persistent, runs handed out by the same counter.
@@ -325,11 +266,6 @@ static void launch_gather(const bls_plan_t *pl)
             configured = smem;
         }
         bls_gather_hot_kernel<LANES, DT><<<pl->sm_count, 768, smem, pl->stream>>>(p, R, rpc);
-    } else if (pl->serve_n_ids == (long long)p.P * p.T * p.b) {
-        // exactly one ID per bag on average: most likely a one-hot iteration (the kernel checks what the router found)
-        const long long want1 = ((long long)p.NI * p.P * p.b + 4 * (256 / LANES) - 1) / (4 * (256 / LANES));
-        const int blocks1 = (int)(want1 < 1 ? 1 : (want1 > pl->sm_count * 3 ? pl->sm_count * 3 : want1));
-        bls_gather_onehot_kernel<LANES, DT><<<blocks1, 256, 0, pl->stream>>>(p, R, rpc, (int)n_runs);
     } else
         bls_gather_pool_kernel<LANES, DT, U><<<blocks, 256, 0, pl->stream>>>(p, R, rpc, (int)n_runs);
 }

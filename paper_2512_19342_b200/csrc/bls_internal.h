@@ -67,7 +67,6 @@ struct BlsDev {
     unsigned long long wait_limit_ns;
     long long max_lag;                            // max over time of newest posted - oldest incomplete
     int status;                                   // OR of BLS_ST_* bits
-    int onehot[BLS_MAX_SLOTS];                    // table-wise: every bag of the iteration in this slot has exactly one ID
     int work_ctr;                                 // next run of the gather kernel (reset by the gate)
     int done_ctr;                                 // blocks of the wave's last kernel that have finished
     int small_ctr;                                // blocks of the fused small-iteration kernel that have finished (its last block resets it)
@@ -161,8 +160,6 @@ struct bls_plan {
     int bags_per_run;             // gather kernel: consecutive sub-bags streamed by one lane group
     int rows_in_flight;           // gather kernel: row loads per batch (4 or 8)
     long long *h_rows;            // host copy of the table heights
-    long long n_ids_of[BLS_MAX_SLOTS];   // IDs of the iteration in each slot (host copy)
-    long long serve_n_ids;        // IDs of the iteration the next gather launch answers (-1 = unknown)
     int ring_used;                // the loop in progress has used the ring kernel: its drain does too (ranks may be behind)
     int ring_mode;                // persistent ring kernel: -1 only with injected delays, 0 also for small iterations, 1 always
     int ring_blocks_per_sm;       // resident blocks of the ring kernel per SM (0 = not queried yet)

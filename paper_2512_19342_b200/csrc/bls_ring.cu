@@ -40,7 +40,6 @@ __device__ __forceinline__ void gate_warp(const BlsParams &p, int mode, long lon
         d->in_ids[slot] = ids;
         d->in_off[slot] = off;
         d->in_n[slot] = n_ids;
-        d->onehot[slot] = 1;                            // the router's copy kernel clears it when it meets a bag of another length
     }
     __syncwarp();
 

@@ -35,17 +35,15 @@ __device__ __forceinline__ int tw_copy_ctx(const BlsParams &p, const RouteCtx &c
     const long long g0 = ((long long)src * p.T + t) * p.b;
     const long long off0 = c.off[g0];
     __shared__ int s_lo, s_hi;
-    bool other_length = false;                   // a bag that does not hold exactly one ID
     for (int s = threadIdx.x; s < nb; s += blockDim.x) {
         int st, en;
         if (!bag_range(c, g0 + s0 + s, off0, cn, st, en)) flag(p, BLS_ST_EINVAL);
-        other_length |= en - st != 1;
         int pos = cb + st;
         c.sub_start[(size_t)i * p.b + s0 + s] = pos > p.cap ? p.cap : pos;
         if (s == 0) s_lo = st;
         if (s == nb - 1) s_hi = en;
     }
-    if (__syncthreads_or(other_length) && threadIdx.x == 0) p.dev->onehot[c.slot] = 0;   // (the barrier also publishes s_lo, s_hi)
+    __syncthreads();                             // s_lo, s_hi
     const unsigned rows = (unsigned)p.tab[t].rows;
     const int lo = s_lo, hi = max(s_lo, s_hi);
     const int *in = c.ids + off0;
